@@ -1,0 +1,179 @@
+/*
+ * libfda - Federated Dynamic Averaging (FDA) monitoring and synchronisation on one GPU.
+ *
+ * The K workers of FDA are K rows of one K x d float32 tensor that lives in the memory of
+ * a single device.  Each round the caller runs
+ *
+ *   fda_local_state      -> S^(k) = (||u^(k)||^2, <xi,u^(k)>, sk(u^(k))),  u^(k) = w^(k) - w_t0
+ *   fda_combine_estimate -> S-bar = mean_k S^(k), H(S-bar), trigger = (H > Theta)
+ *   fda_average_models   -> w^(k) := w-bar = mean_k w^(k)  (and w_t0 := w-bar) if triggered
+ *
+ * which are lines 6-9 of Algorithm 1 of the FDA paper (Section 3) with the two AllReduce
+ * steps replaced by reductions over rows in device memory.
+ *
+ * Conventions
+ *   - plain C ABI; every function returns an fda_status and never throws or aborts;
+ *   - unless a parameter says "host", pointers are DEVICE pointers to memory owned by the
+ *     caller; the library never frees or reallocates caller memory;
+ *   - the context owns its own device scratch (hash table, per-block partial sums);
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); calls
+ *     enqueue work and return, unless stated otherwise;
+ *   - arguments are validated on the host before anything is launched; an invalid call
+ *     launches nothing and leaves its outputs untouched;
+ *   - one context serves one stream at a time (calls on the same context must not overlap
+ *     on the device, because they share the context's scratch).
+ *
+ * State layout (float32, state_len = 2 + l*m per worker, row-major):
+ *   [0]              ||u^(k)||^2                                   (Section 3, local state)
+ *   [1]              <xi, u^(k)>                                   (Theorem 2, LinearFDA)
+ *   [2 + i*m + c]    cell c of row i of the AMS sketch sk(u^(k))   (Theorem 1, SketchFDA)
+ */
+#ifndef FDA_H_
+#define FDA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fda_ctx fda_ctx; /* opaque, library-owned */
+
+typedef enum {
+    FDA_OK = 0,
+    FDA_ERR_INVALID_ARG = 1, /* NULL pointer, size out of range, bad flag               */
+    FDA_ERR_UNSUPPORTED = 2, /* valid request the kernels cannot serve (sketch too big) */
+    FDA_ERR_CUDA = 3,        /* a CUDA runtime call failed; see fda_last_error          */
+    FDA_ERR_NOMEM = 4        /* host or device allocation failed                        */
+} fda_status;
+
+/* Which parts of the local state fda_local_state computes; parts not asked for are
+ * written as 0. */
+enum { FDA_STATE_NORM = 1, FDA_STATE_LINEAR = 2, FDA_STATE_SKETCH = 4 };
+/* Estimator used by fda_combine_estimate. */
+enum { FDA_VARIANT_LINEAR = 0, FDA_VARIANT_SKETCH = 1 };
+/* fda_average_models flags. */
+enum {
+    FDA_AVG_BROADCAST = 1,     /* also overwrite every w^(k) with w-bar (in-place sync) */
+    FDA_AVG_UNCONDITIONAL = 2  /* ignore the trigger flag of the estimate               */
+};
+
+#define FDA_MAX_ROWS 16 /* largest supported number of sketch rows l */
+
+/* Result of fda_combine_estimate. */
+typedef struct {
+    float mean_sq_norm;        /* (1/K) sum_k ||u^(k)||^2                              */
+    float est_sq_norm_of_mean; /* the estimate of ||u-bar||^2 that H subtracts         */
+    float H;                   /* variance over-estimate                               */
+    float theta;               /* the threshold it was compared with                   */
+    int32_t trigger;           /* 1 if H > theta (strictly), else 0                    */
+    int32_t l;                 /* number of valid entries of row_sq_norm               */
+    float row_sq_norm[FDA_MAX_ROWS]; /* ||row i of the averaged sketch||^2             */
+} fda_estimate;
+
+/*
+ * Create a context on CUDA device `device` for sketches of l rows x m columns.
+ *   hash_coeffs  HOST pointer to 6*l uint64 values, per row {a, b, c3, c2, c1, c0}, each in
+ *                [0, 2^61-2], a != 0 and c3 != 0.  They define the AMS hash family
+ *                (Section 3.1 cites the sketch but prints no family; this is the classical
+ *                2-wise bucket / 4-wise sign construction over p = 2^61-1):
+ *                  bucket_i(j) = ((a*j + b) mod p) mod m
+ *                  sign_i(j)   = +1 if ((((c3*j + c2)*j + c1)*j + c0) mod p) is even, else -1
+ *                May be NULL when l == 0 (a context without sketch: state_len = 2).
+ *   d_max, K_max largest model dimension / worker count later calls will use; they size
+ *                the context's scratch (2*l bytes of hash table per index, plus partial
+ *                sums).  Blocking: allocates, fills the hash table, synchronises.
+ * Errors: INVALID_ARG (out == NULL, l < 0 or > FDA_MAX_ROWS, m < 1 or > 32768 with l > 0,
+ * d_max < 1 or >= 2^31, K_max < 1, coefficient out of range), UNSUPPORTED (l*m too large
+ * for the shared-memory bins), NOMEM, CUDA.
+ */
+fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
+                      int64_t d_max, int K_max);
+
+/* Free the context and its scratch.  Blocking (synchronises the device). NULL is a no-op. */
+fda_status fda_destroy(fda_ctx *ctx);
+
+/* Floats per worker state: 2 + l*m. 0 if ctx == NULL. */
+size_t fda_state_len(const fda_ctx *ctx);
+
+/* HOST string describing the last error on this context (empty if none). */
+const char *fda_last_error(const fda_ctx *ctx);
+
+/*
+ * Local states of all K workers in one pass over w (Section 3: local drift, local state;
+ * Section 3.1: sk(.); Section 3.2: <xi,u>).
+ *   w           K rows of d floats, row k at w + k*row_stride (row_stride >= d, elements)
+ *   w_t0        d floats, model after the last synchronisation
+ *   xi          d floats (unit vector of LinearFDA) or NULL; used only with FDA_STATE_LINEAR
+ *   flags       OR of FDA_STATE_*; FDA_STATE_SKETCH needs l > 0
+ *   states      out, K x state_len floats
+ * Any alignment of w, w_t0, xi is accepted; 16-byte aligned pointers with row_stride a
+ * multiple of 4 take the vector path.  Errors: INVALID_ARG (NULL, K < 1 or > K_max, d < 1
+ * or > d_max, row_stride < d, unknown flag, SKETCH without a sketch), CUDA.
+ */
+fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
+                           const float *w_t0, const float *xi, uint32_t flags, float *states,
+                           void *stream);
+
+/*
+ * Average the K states and evaluate the variance over-estimate (Algorithm 1 lines 7-8).
+ *   FDA_VARIANT_SKETCH: H = S-bar[0] - median_i ||row_i(S-bar sketch)||^2 / (1 + epsilon)
+ *                       (Theorem 1; the median of an even number of rows is the mean of
+ *                       the two middle values);
+ *   FDA_VARIANT_LINEAR: H = S-bar[0] - S-bar[1]^2                            (Theorem 2).
+ *   trigger = (H > theta).  Accumulation is in fp64, results are rounded to fp32.
+ *   states      K x state_len floats (as written by fda_local_state)
+ *   est_dev     out, DEVICE fda_estimate
+ *   est_host    out, HOST fda_estimate or NULL.  If not NULL the call copies the result
+ *               and synchronises `stream` before returning.
+ * Errors: INVALID_ARG (NULL, K < 1 or > K_max, bad variant, SKETCH variant with l == 0,
+ * epsilon <= -1 or not finite, theta not finite), CUDA.
+ */
+fda_status fda_combine_estimate(fda_ctx *ctx, const float *states, int K, int variant,
+                                float epsilon, float theta, fda_estimate *est_dev,
+                                fda_estimate *est_host, void *stream);
+
+/*
+ * Synchronise: w-bar[j] = (1/K) sum_k w^(k)[j] (fp32, summed in the order k = 0..K-1), then
+ * w_t0 := w-bar and, with FDA_AVG_BROADCAST, every w^(k) := w-bar in place (Section 3,
+ * "Workers synchronize by executing AllReduce"; Algorithm 1 line 9).
+ *   est_dev     DEVICE fda_estimate whose `trigger` gates the whole operation on the
+ *               device (nothing is read or written when it is 0); NULL or
+ *               FDA_AVG_UNCONDITIONAL averages always.
+ * Errors: INVALID_ARG (NULL w or w_t0, K < 1, d < 1, row_stride < d, unknown flag), CUDA.
+ */
+fda_status fda_average_models(fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                              float *w_t0, const fda_estimate *est_dev, uint32_t flags,
+                              void *stream);
+
+/*
+ * One whole round on HOST buffers: copies w, w_t0 and xi to device staging owned by the
+ * context (allocated on first use for K_max x d_max), runs fda_local_state,
+ * fda_combine_estimate and fda_average_models (FDA_AVG_BROADCAST, gated by the trigger) and
+ * copies back the states, the estimate and - only if the round triggered - the averaged
+ * model into w_t0_host (and into every row of w_host when `avg_flags` has
+ * FDA_AVG_BROADCAST).  Blocking.  Pinned host buffers make the copies asynchronous to the
+ * host but the call still waits for completion.
+ *   states_host  out, K x state_len floats, may be NULL
+ *   est_host     out, required
+ * Errors: as the three calls above, plus NOMEM for the staging buffers.
+ */
+fda_status fda_round_host(fda_ctx *ctx, float *w_host, int64_t row_stride, int K, int64_t d,
+                          float *w_t0_host, const float *xi_host, uint32_t state_flags,
+                          int variant, float epsilon, float theta, uint32_t avg_flags,
+                          float *states_host, fda_estimate *est_host, void *stream);
+
+/*
+ * Hash dump for parity checks: for indices j0 .. j0+n-1 and every row i < l writes
+ * buckets[i*n + t] = bucket_i(j0+t) and signs[i*n + t] = sign_i(j0+t) (+1 / -1), evaluated
+ * directly from the coefficients (not read from the context's table).
+ * Errors: INVALID_ARG (NULL, l == 0, j0 < 0, n < 1, j0 + n > 2^31), CUDA.
+ */
+fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets,
+                          int8_t *signs, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDA_H_ */

@@ -1,0 +1,212 @@
+"""ctypes binding of libfda (see include/fda.h for the contract of every call).
+
+The functions keep the names of the C entry points (``fda_local_state`` ...) as methods of
+:class:`FdaContext`; they pass ``tensor.data_ptr()`` and the current torch stream through and
+do nothing else.  There is no fallback: if the shared library is missing or a call fails,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+FDA_STATE_NORM, FDA_STATE_LINEAR, FDA_STATE_SKETCH = 1, 2, 4
+FDA_VARIANT_LINEAR, FDA_VARIANT_SKETCH = 0, 1
+FDA_AVG_BROADCAST, FDA_AVG_UNCONDITIONAL = 1, 2
+FDA_MAX_ROWS = 16
+
+_STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "FDA_ERR_CUDA",
+           4: "FDA_ERR_NOMEM"}
+
+EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state",
+           "fda_combine_estimate", "fda_average_models", "fda_round_host", "fda_debug_hash")
+
+
+class FdaError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__("%s failed with %s%s" % (where, _STATUS.get(status, status),
+                                                   (": " + detail) if detail else ""))
+
+
+class Estimate(ctypes.Structure):
+    """Mirror of ``fda_estimate``."""
+    _fields_ = [("mean_sq_norm", ctypes.c_float), ("est_sq_norm_of_mean", ctypes.c_float),
+                ("H", ctypes.c_float), ("theta", ctypes.c_float), ("trigger", ctypes.c_int32),
+                ("l", ctypes.c_int32), ("row_sq_norm", ctypes.c_float * FDA_MAX_ROWS)]
+
+    def as_dict(self):
+        return {"mean_sq": self.mean_sq_norm, "est": self.est_sq_norm_of_mean, "H": self.H,
+                "theta": self.theta, "trigger": bool(self.trigger),
+                "rows": np.array(self.row_sq_norm[:self.l], dtype=np.float32)}
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfda.so")
+
+
+def load_library():
+    """Load libfda.so from the package directory (never from anywhere else)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise FdaError(3, "load_library", "%s not found - run `python -m paper_2405_20988_b200.build`" % path)
+    lib = ctypes.CDLL(path)
+    vp, i64, c_int, u32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint32, ctypes.c_float
+    lib.fda_create.argtypes = [ctypes.POINTER(vp), c_int, c_int, c_int, vp, i64, c_int]
+    lib.fda_destroy.argtypes = [vp]
+    lib.fda_state_len.argtypes = [vp]
+    lib.fda_state_len.restype = ctypes.c_size_t
+    lib.fda_last_error.argtypes = [vp]
+    lib.fda_last_error.restype = ctypes.c_char_p
+    lib.fda_local_state.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
+    lib.fda_combine_estimate.argtypes = [vp, vp, c_int, c_int, f32, f32, vp, vp, vp]
+    lib.fda_average_models.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp]
+    lib.fda_round_host.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, c_int, f32, f32, u32, vp, vp, vp]
+    lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
+    for name in ("fda_create", "fda_destroy", "fda_local_state", "fda_combine_estimate",
+                 "fda_average_models", "fda_round_host", "fda_debug_hash"):
+        getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+def _dev_ptr(t, dtype=None, name="tensor"):
+    """Device pointer of a CUDA torch tensor (None passes NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("%s must have dtype %s" % (name, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _rows(w, name="w"):
+    """(pointer, row_stride, K, d) of a 2-D float32 tensor/array whose rows are contiguous."""
+    if w.dim() != 2 or (w.shape[1] > 1 and w.stride(1) != 1):
+        raise ValueError("%s must be 2-D with contiguous rows" % name)
+    K, d = w.shape
+    stride = w.stride(0) if K > 1 else max(w.stride(0), d)
+    return stride, K, d
+
+
+class FdaContext:
+    """Owner of an ``fda_ctx``.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, l: int, m: int, hash_coeffs, d_max: int, K_max: int, device: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        coeffs = None
+        if l > 0:
+            coeffs = np.ascontiguousarray(hash_coeffs, dtype=np.uint64).reshape(-1)
+            if coeffs.size != 6 * l:
+                raise ValueError("hash_coeffs must hold 6*l values")
+        self._coeffs = coeffs
+        ptr = coeffs.ctypes.data_as(ctypes.c_void_p) if coeffs is not None else None
+        st = self._lib.fda_create(ctypes.byref(self._h), device, l, m, ptr, d_max, K_max)
+        if st != 0:
+            self._h = ctypes.c_void_p()
+            raise FdaError(st, "fda_create")
+        self.l, self.m, self.d_max, self.K_max, self.device = l, m if l > 0 else 0, d_max, K_max, device
+
+    # -- helpers ---------------------------------------------------------------------------
+    def _check(self, st: int, where: str):
+        if st != 0:
+            raise FdaError(st, where, self._lib.fda_last_error(self._h).decode())
+
+    @property
+    def state_len(self) -> int:
+        return int(self._lib.fda_state_len(self._h))
+
+    def fda_last_error(self) -> str:
+        return self._lib.fda_last_error(self._h).decode()
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.fda_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- the C entry points ----------------------------------------------------------------
+    def fda_local_state(self, w, w_t0, xi, flags: int, states, stream=None):
+        """states[K, state_len] <- local states of the K rows of w (device tensors)."""
+        import torch
+        stride, K, d = _rows(w)
+        st = self._lib.fda_local_state(self._h, _dev_ptr(w, torch.float32, "w"), stride, K, d,
+                                       _dev_ptr(w_t0, torch.float32, "w_t0"),
+                                       _dev_ptr(xi, torch.float32, "xi"), flags,
+                                       _dev_ptr(states, torch.float32, "states"), _stream_ptr(stream))
+        self._check(st, "fda_local_state")
+
+    def fda_combine_estimate(self, states, K: int, variant: int, epsilon: float, theta: float,
+                             est_dev, want_host: bool = True, stream=None):
+        """est_dev: uint8 CUDA tensor of sizeof(fda_estimate) bytes.  Returns an Estimate
+        (host copy, synchronises the stream) when ``want_host``, else None."""
+        import torch
+        host = Estimate() if want_host else None
+        st = self._lib.fda_combine_estimate(self._h, _dev_ptr(states, torch.float32, "states"), K,
+                                            variant, epsilon, theta, _dev_ptr(est_dev, torch.uint8, "est_dev"),
+                                            ctypes.byref(host) if host is not None else None,
+                                            _stream_ptr(stream))
+        self._check(st, "fda_combine_estimate")
+        return host
+
+    def fda_average_models(self, w, w_t0, est_dev, flags: int, stream=None):
+        import torch
+        stride, K, d = _rows(w)
+        st = self._lib.fda_average_models(self._h, _dev_ptr(w, torch.float32, "w"), stride, K, d,
+                                          _dev_ptr(w_t0, torch.float32, "w_t0"),
+                                          _dev_ptr(est_dev, torch.uint8, "est_dev"), flags,
+                                          _stream_ptr(stream))
+        self._check(st, "fda_average_models")
+
+    def fda_round_host(self, w_host, w_t0_host, xi_host, state_flags: int, variant: int,
+                       epsilon: float, theta: float, avg_flags: int, states_host=None, stream=None):
+        """Whole round on HOST tensors (CPU torch tensors, ideally pinned).  Returns Estimate."""
+        stride, K, d = _rows(w_host, "w_host")
+        est = Estimate()
+
+        def hp(t):
+            return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+        st = self._lib.fda_round_host(self._h, hp(w_host), stride, K, d, hp(w_t0_host), hp(xi_host),
+                                      state_flags, variant, epsilon, theta, avg_flags,
+                                      hp(states_host), ctypes.byref(est), _stream_ptr(stream))
+        self._check(st, "fda_round_host")
+        return est
+
+    def fda_debug_hash(self, j0: int, n: int, buckets, signs, stream=None):
+        """buckets: uint16[l, n] (torch.int16 storage is accepted), signs: int8[l, n]."""
+        st = self._lib.fda_debug_hash(self._h, j0, n, ctypes.c_void_p(buckets.data_ptr()),
+                                      ctypes.c_void_p(signs.data_ptr()), _stream_ptr(stream))
+        self._check(st, "fda_debug_hash")
+
+    @staticmethod
+    def new_estimate_buffer(device="cuda"):
+        import torch
+        return torch.zeros(ctypes.sizeof(Estimate), dtype=torch.uint8, device=device)

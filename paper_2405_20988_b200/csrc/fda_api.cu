@@ -1,0 +1,282 @@
+// C ABI of libfda: context management, argument validation, stream plumbing.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "fda_internal.h"
+
+namespace {
+
+constexpr uint64_t kP61 = (1ull << 61) - 1;
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; prev = -1; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+fda_status fail(fda_ctx *ctx, fda_status st, const char *what)
+{
+    if (ctx) ctx->err = what;
+    return st;
+}
+
+fda_status fail_cuda(fda_ctx *ctx, cudaError_t e, const char *where)
+{
+    if (ctx) {
+        ctx->err = std::string(where) + ": " + cudaGetErrorString(e);
+    }
+    return e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;
+}
+
+void free_device(fda_ctx *ctx)
+{
+    cudaFree(ctx->coeffs_dev);
+    cudaFree(ctx->tab);
+    cudaFree(ctx->part_sk);
+    cudaFree(ctx->part_np);
+    cudaFree(ctx->stage_w);
+    cudaFree(ctx->stage_w_t0);
+    cudaFree(ctx->stage_xi);
+    cudaFree(ctx->stage_states);
+    cudaFree(ctx->stage_est);
+}
+
+bool finite_f(float v) { return std::isfinite(v); }
+
+}  // namespace
+
+extern "C" {
+
+fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
+                      int64_t d_max, int K_max)
+{
+    if (!out) return FDA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (l < 0 || l > FDA_MAX_ROWS) return FDA_ERR_INVALID_ARG;
+    if (l > 0 && (m < 1 || m > 32768 || !hash_coeffs)) return FDA_ERR_INVALID_ARG;
+    if (d_max < 1 || d_max >= (int64_t)1 << 31 || K_max < 1) return FDA_ERR_INVALID_ARG;
+    for (int i = 0; i < 6 * l; ++i) {
+        if (hash_coeffs[i] >= kP61) return FDA_ERR_INVALID_ARG;
+        if ((i % 6 == 0 || i % 6 == 2) && hash_coeffs[i] == 0) return FDA_ERR_INVALID_ARG;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+        cudaGetLastError();
+        return FDA_ERR_CUDA;
+    }
+    fda_ctx *ctx = new (std::nothrow) fda_ctx();
+    if (!ctx) return FDA_ERR_NOMEM;
+    ctx->device = device;
+    ctx->l = l;
+    ctx->m = l > 0 ? m : 0;
+    ctx->lm = ctx->l * ctx->m;
+    ctx->d_max = d_max;
+    ctx->K_max = K_max;
+    for (int i = 0; i < 6 * l; ++i) ctx->coeffs_host[i] = hash_coeffs[i];
+
+    DeviceGuard guard(device);
+    cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e != cudaSuccess) { delete ctx; return FDA_ERR_CUDA; }
+
+    fda_setup_local_state(ctx);
+    if (l > 0 && ctx->columns < 1) { delete ctx; return FDA_ERR_UNSUPPORTED; }
+
+    ctx->max_blocks = ctx->n_sm * 4;
+    ctx->tab_stride = (d_max + 63) / 64 * 64;
+    ctx->part_sk_floats = l > 0 ? (size_t)ctx->n_sm * ctx->lm * ctx->columns : 0;
+    if (l > 0) {
+        e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * (size_t)ctx->max_blocks * 32 * 2);
+    if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        const fda_status st = e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;
+        cudaGetLastError();
+        free_device(ctx);
+        delete ctx;
+        return st;
+    }
+    *out = ctx;
+    return FDA_OK;
+}
+
+fda_status fda_destroy(fda_ctx *ctx)
+{
+    if (!ctx) return FDA_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    free_device(ctx);
+    delete ctx;
+    return FDA_OK;
+}
+
+size_t fda_state_len(const fda_ctx *ctx) { return ctx ? 2 + (size_t)ctx->lm : 0; }
+
+const char *fda_last_error(const fda_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
+                           const float *w_t0, const float *xi, uint32_t flags, float *states,
+                           void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!w || !w_t0 || !states) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: null pointer");
+    if (K < 1 || K > ctx->K_max) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: K out of range");
+    if (d < 1 || d > ctx->d_max) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: d out of range");
+    if (row_stride < d) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: row_stride < d");
+    if (flags & ~(uint32_t)(FDA_STATE_NORM | FDA_STATE_LINEAR | FDA_STATE_SKETCH))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: unknown flag");
+    if ((flags & FDA_STATE_SKETCH) && ctx->l == 0)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_local_state: context has no sketch");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_local_state: cannot select device");
+    cudaError_t e = fda_launch_local_state(ctx, w, row_stride, K, d, w_t0, xi, flags, states,
+                                           (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_local_state");
+    return FDA_OK;
+}
+
+fda_status fda_combine_estimate(fda_ctx *ctx, const float *states, int K, int variant,
+                                float epsilon, float theta, fda_estimate *est_dev,
+                                fda_estimate *est_host, void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!states || !est_dev) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_combine_estimate: null pointer");
+    if (K < 1 || K > ctx->K_max) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_combine_estimate: K out of range");
+    if (variant != FDA_VARIANT_LINEAR && variant != FDA_VARIANT_SKETCH)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_combine_estimate: bad variant");
+    if (variant == FDA_VARIANT_SKETCH && ctx->l == 0)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_combine_estimate: context has no sketch");
+    if (!finite_f(epsilon) || epsilon <= -1.0f || !finite_f(theta))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_combine_estimate: epsilon or theta out of range");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_combine_estimate: cannot select device");
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = fda_launch_combine(ctx, states, K, variant, epsilon, theta, est_dev, s);
+    if (e == cudaSuccess && est_host) {
+        e = cudaMemcpyAsync(est_host, est_dev, sizeof(fda_estimate), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    }
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_combine_estimate");
+    return FDA_OK;
+}
+
+fda_status fda_average_models(fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                              float *w_t0, const fda_estimate *est_dev, uint32_t flags,
+                              void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!w || !w_t0) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models: null pointer");
+    if (K < 1 || d < 1 || row_stride < d)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models: size out of range");
+    if (flags & ~(uint32_t)(FDA_AVG_BROADCAST | FDA_AVG_UNCONDITIONAL))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models: unknown flag");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_average_models: cannot select device");
+    cudaError_t e = fda_launch_average(ctx, w, row_stride, K, d, w_t0, est_dev, flags,
+                                       (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_average_models");
+    return FDA_OK;
+}
+
+fda_status fda_round_host(fda_ctx *ctx, float *w_host, int64_t row_stride, int K, int64_t d,
+                          float *w_t0_host, const float *xi_host, uint32_t state_flags,
+                          int variant, float epsilon, float theta, uint32_t avg_flags,
+                          float *states_host, fda_estimate *est_host, void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!w_host || !w_t0_host || !est_host)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_round_host: null pointer");
+    if (K < 1 || K > ctx->K_max || d < 1 || d > ctx->d_max || row_stride < d)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_round_host: size out of range");
+    if (avg_flags & ~(uint32_t)(FDA_AVG_BROADCAST | FDA_AVG_UNCONDITIONAL))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_round_host: unknown flag");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_round_host: cannot select device");
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t slen = fda_state_len(ctx);
+    cudaError_t e = cudaSuccess;
+    if (!ctx->stage_w) {
+        ctx->stage_stride = (ctx->d_max + 31) / 32 * 32;
+        e = cudaMalloc(&ctx->stage_w, sizeof(float) * (size_t)ctx->K_max * ctx->stage_stride);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->stage_w_t0, sizeof(float) * ctx->stage_stride);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->stage_xi, sizeof(float) * ctx->stage_stride);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->stage_states, sizeof(float) * (size_t)ctx->K_max * slen);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->stage_est, sizeof(fda_estimate));
+        if (e != cudaSuccess) {
+            cudaFree(ctx->stage_w); cudaFree(ctx->stage_w_t0); cudaFree(ctx->stage_xi);
+            cudaFree(ctx->stage_states); cudaFree(ctx->stage_est);
+            ctx->stage_w = ctx->stage_w_t0 = ctx->stage_xi = ctx->stage_states = nullptr;
+            ctx->stage_est = nullptr;
+            cudaGetLastError();
+            return fail_cuda(ctx, e, "fda_round_host: staging allocation");
+        }
+    }
+    const int64_t sst = ctx->stage_stride;
+    e = cudaMemcpy2DAsync(ctx->stage_w, sizeof(float) * sst, w_host, sizeof(float) * row_stride,
+                          sizeof(float) * d, (size_t)K, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(ctx->stage_w_t0, w_t0_host, sizeof(float) * d, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && xi_host)
+        e = cudaMemcpyAsync(ctx->stage_xi, xi_host, sizeof(float) * d, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_round_host: host-to-device copy");
+
+    fda_status st = fda_local_state(ctx, ctx->stage_w, sst, K, d, ctx->stage_w_t0,
+                                    xi_host ? ctx->stage_xi : nullptr, state_flags,
+                                    ctx->stage_states, stream);
+    if (st != FDA_OK) return st;
+    st = fda_combine_estimate(ctx, ctx->stage_states, K, variant, epsilon, theta, ctx->stage_est,
+                              est_host, stream);          // synchronises: est_host is valid
+    if (st != FDA_OK) return st;
+    if (states_host) {
+        e = cudaMemcpyAsync(states_host, ctx->stage_states, sizeof(float) * (size_t)K * slen,
+                            cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_round_host: states copy");
+    }
+    const bool fire = (avg_flags & FDA_AVG_UNCONDITIONAL) || est_host->trigger != 0;
+    if (fire) {
+        st = fda_average_models(ctx, ctx->stage_w, sst, K, d, ctx->stage_w_t0, nullptr,
+                                (avg_flags & FDA_AVG_BROADCAST) | FDA_AVG_UNCONDITIONAL, stream);
+        if (st != FDA_OK) return st;
+        e = cudaMemcpyAsync(w_t0_host, ctx->stage_w_t0, sizeof(float) * d, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && (avg_flags & FDA_AVG_BROADCAST))
+            e = cudaMemcpy2DAsync(w_host, sizeof(float) * row_stride, ctx->stage_w, sizeof(float) * sst,
+                                  sizeof(float) * d, (size_t)K, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_round_host: device-to-host copy");
+    }
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_round_host: synchronize");
+    return FDA_OK;
+}
+
+fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets, int8_t *signs,
+                          void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!buckets || !signs || ctx->l == 0 || j0 < 0 || n < 1 || j0 + n > ((int64_t)1 << 31))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_debug_hash: argument out of range");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_debug_hash: cannot select device");
+    cudaError_t e = fda_launch_debug_hash(ctx, j0, n, buckets, signs, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_debug_hash");
+    return FDA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+// K-way model average (Section 3: "Workers synchronize by executing AllReduce", Algorithm 1
+// line 9): w-bar = (1/K) sum_k w^(k), written to w_t0 and, when broadcasting, to every row.
+// Bandwidth-bound streaming kernel; the whole launch is predicated on the trigger word of
+// the device-side estimate so that no host round trip is needed between the two calls.
+#include "fda_internal.h"
+
+namespace {
+
+constexpr int kBatch = 8;   // rows loaded before they are summed (loads in flight per thread)
+
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+k_average(float *w, int64_t row_stride, int K, int64_t d, float *__restrict__ w_t0,
+          const fda_estimate *est, int broadcast)
+{
+    if (est != nullptr && est->trigger == 0) return;
+    const float inv_k = 1.0f / (float)K;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (VEC) {
+        const int64_t nq = d / 4;
+        for (int64_t q = t0; q < nq; q += nthreads) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k0 = 0; k0 < K; k0 += kBatch) {
+                float4 v[kBatch];
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b)
+                    if (k0 + b < K)
+                        v[b] = *reinterpret_cast<const float4 *>(w + (size_t)(k0 + b) * row_stride + q * 4);
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b)
+                    if (k0 + b < K) { acc.x += v[b].x; acc.y += v[b].y; acc.z += v[b].z; acc.w += v[b].w; }
+            }
+            acc.x *= inv_k; acc.y *= inv_k; acc.z *= inv_k; acc.w *= inv_k;
+            *reinterpret_cast<float4 *>(w_t0 + q * 4) = acc;
+            if (broadcast)
+                for (int k = 0; k < K; ++k)
+                    *reinterpret_cast<float4 *>(w + (size_t)k * row_stride + q * 4) = acc;
+        }
+    }
+    // scalar path: everything when !VEC, the d % 4 tail otherwise
+    const int64_t begin = VEC ? (d / 4) * 4 : 0;
+    for (int64_t j = begin + t0; j < d; j += nthreads) {
+        float acc = 0.f;
+        for (int k = 0; k < K; ++k) acc += w[(size_t)k * row_stride + j];
+        acc *= inv_k;
+        w_t0[j] = acc;
+        if (broadcast)
+            for (int k = 0; k < K; ++k) w[(size_t)k * row_stride + j] = acc;
+    }
+}
+
+}  // namespace
+
+cudaError_t fda_launch_average(const fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                               float *w_t0, const fda_estimate *est_dev, uint32_t flags,
+                               cudaStream_t s)
+{
+    const bool vec = ((((uintptr_t)w | (uintptr_t)w_t0) & 15u) == 0) && (row_stride % 4 == 0);
+    const fda_estimate *gate = (flags & FDA_AVG_UNCONDITIONAL) ? nullptr : est_dev;
+    const int broadcast = (flags & FDA_AVG_BROADCAST) ? 1 : 0;
+    const int threads = 256;
+    int64_t work = vec ? (d + 3) / 4 : d;
+    int64_t blocks = (work + threads - 1) / threads;
+    const int64_t cap = (int64_t)ctx->n_sm * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (vec) k_average<true><<<(unsigned)blocks, threads, 0, s>>>(w, row_stride, K, d, w_t0, gate, broadcast);
+    else     k_average<false><<<(unsigned)blocks, threads, 0, s>>>(w, row_stride, K, d, w_t0, gate, broadcast);
+    return cudaGetLastError();
+}

@@ -1,0 +1,53 @@
+// Internal declarations shared by the translation units of libfda (not installed).
+#ifndef FDA_INTERNAL_H_
+#define FDA_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string>
+
+#include "../../include/fda.h"
+
+// Hash-table entry: bits 0..14 bucket, bit 15 set when the sign is -1.
+#define FDA_TAB_SIGN_BIT 0x8000u
+
+struct fda_ctx {
+    int device = 0;
+    int n_sm = 0;
+    int smem_optin = 0;        // largest dynamic shared memory per block (bytes)
+    int l = 0, m = 0, lm = 0;
+    int64_t d_max = 0;
+    int K_max = 0;
+    // sketch geometry (valid when l > 0)
+    int columns = 0;           // lane-private columns per cell in the shared-memory bins
+    // device scratch
+    uint64_t *coeffs_dev = nullptr;   // 6*l
+    uint16_t *tab = nullptr;          // l planes of tab_stride entries
+    int64_t tab_stride = 0;
+    float *part_sk = nullptr;         // per-block sketch partials
+    size_t part_sk_floats = 0;
+    double *part_np = nullptr;        // per-block (norm, projection) partials
+    int max_blocks = 0;
+    // staging for fda_round_host (lazy)
+    float *stage_w = nullptr, *stage_w_t0 = nullptr, *stage_xi = nullptr, *stage_states = nullptr;
+    fda_estimate *stage_est = nullptr;
+    int64_t stage_stride = 0;
+    uint64_t coeffs_host[6 * FDA_MAX_ROWS] = {0};
+    std::string err;
+};
+
+// ---- launchers (each returns the cudaError_t of its launches) -------------------------
+cudaError_t fda_launch_build_table(const fda_ctx *ctx, cudaStream_t s);
+cudaError_t fda_launch_debug_hash(const fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets,
+                                  int8_t *signs, cudaStream_t s);
+cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                   int64_t d, const float *w_t0, const float *xi, uint32_t flags,
+                                   float *states, cudaStream_t s);
+cudaError_t fda_setup_local_state(fda_ctx *ctx);   // opt-in shared memory, pick geometry
+cudaError_t fda_launch_combine(const fda_ctx *ctx, const float *states, int K, int variant,
+                               float epsilon, float theta, fda_estimate *est_dev, cudaStream_t s);
+cudaError_t fda_launch_average(const fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                               float *w_t0, const fda_estimate *est_dev, uint32_t flags,
+                               cudaStream_t s);
+
+#endif
