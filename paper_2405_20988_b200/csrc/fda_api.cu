@@ -44,6 +44,7 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->tab);
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
+    cudaFree(ctx->err_flag);
     cudaFree(ctx->stage_w);
     cudaFree(ctx->stage_w_t0);
     cudaFree(ctx->stage_xi);
@@ -96,7 +97,7 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
 
     ctx->max_blocks = ctx->n_sm * 4;
     ctx->tab_stride = (d_max + 63) / 64 * 64;
-    ctx->part_sk_floats = l > 0 ? (size_t)ctx->n_sm * ctx->lm * ctx->columns : 0;
+    ctx->part_sk_floats = l > 0 ? (size_t)ctx->n_sm * ctx->lm * 32 : 0;
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
@@ -105,6 +106,8 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
             e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * (size_t)ctx->max_blocks * 32 * 2);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->err_flag, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->err_flag, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -171,8 +174,14 @@ fda_status fda_combine_estimate(fda_ctx *ctx, const float *states, int K, int va
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = fda_launch_combine(ctx, states, K, variant, epsilon, theta, est_dev, s);
     if (e == cudaSuccess && est_host) {
+        unsigned int flag = 0;
         e = cudaMemcpyAsync(est_host, est_dev, sizeof(fda_estimate), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&flag, ctx->err_flag, sizeof(flag), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e == cudaSuccess && flag != 0) {
+            cudaMemsetAsync(ctx->err_flag, 0, sizeof(flag), s);
+            return fail(ctx, FDA_ERR_CUDA, "a device-side wait of an earlier fda_local_state ran out; its states are invalid");
+        }
     }
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_combine_estimate");
     return FDA_OK;

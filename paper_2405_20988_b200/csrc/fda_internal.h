@@ -28,6 +28,7 @@ struct fda_ctx {
     size_t part_sk_floats = 0;
     double *part_np = nullptr;        // per-block (norm, projection) partials
     int max_blocks = 0;
+    unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
     // staging for fda_round_host (lazy)
     float *stage_w = nullptr, *stage_w_t0 = nullptr, *stage_xi = nullptr, *stage_states = nullptr;
     fda_estimate *stage_est = nullptr;
@@ -43,6 +44,9 @@ cudaError_t fda_launch_debug_hash(const fda_ctx *ctx, int64_t j0, int64_t n, uin
 cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s);
+cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, cudaStream_t s);
 cudaError_t fda_setup_local_state(fda_ctx *ctx);   // opt-in shared memory, pick geometry
 cudaError_t fda_launch_combine(const fda_ctx *ctx, const float *states, int K, int variant,
                                float epsilon, float theta, fda_estimate *est_dev, cudaStream_t s);
