@@ -34,7 +34,8 @@ import fda_synth as S  # noqa: E402
 
 METRIC = "FDA local-state+sketch throughput (local state -> estimate -> K-way average)"
 UNIT = "params*workers/s"
-ALL_STATE = 1 | 2 | 4
+SKETCH_STATE = 1 | 4      # SketchFDA local state (Theorem 1): squared norm + AMS sketch
+LINEAR_STATE = 1 | 2      # LinearFDA local state (Theorem 2): squared norm + projection
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
@@ -122,7 +123,7 @@ def oracle_step_on_sample(wl, w_host, w_t0, xi, coeffs, d_sample, threads):
     """One whole step of the CPU oracle on the first d_sample indices of every worker."""
     import oracle
     t0 = time.perf_counter()
-    st = oracle.local_state(w_host[:, :d_sample], w_t0[:d_sample], xi[:d_sample], coeffs, wl.l, wl.m,
+    st = oracle.local_state(w_host[:, :d_sample], w_t0[:d_sample], None, coeffs, wl.l, wl.m,
                             threads=threads)
     est = oracle.combine(st, wl.l, wl.m, 1, wl.epsilon, wl.thetas[-1])
     if est["trigger"]:
@@ -182,7 +183,7 @@ def run_ours(args, rank, world, local_rank):
         w0.copy_(w0_src)
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         ev[0].record(stream)
-        ctx.fda_local_state(w[:, :d], w0, xi, ALL_STATE, states)
+        ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
         ev[1].record(stream)
         ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, eps, theta, est_buf, want_host=False)
         ev[2].record(stream)
@@ -214,6 +215,21 @@ def run_ours(args, rank, world, local_rank):
     est = F.Estimate.from_buffer_copy(bytes(est_buf.cpu().numpy()))
     if not est.trigger:
         raise SystemExit("bench: the round did not trigger; the average was not timed")
+
+    # ---- the LinearFDA flavour of the local-state pass, timed beside the headline step ----
+    w.copy_(w_src)
+    w0.copy_(w0_src)
+    lin_ms = []
+    for it in range(3 + 10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.fda_local_state(w[:, :d], w0, xi, LINEAR_STATE, states)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            lin_ms.append(e0.elapsed_time(e1))
+    lin_ms = float(np.mean(lin_ms))
+    lin_est = ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_LINEAR, eps, theta, est_buf).as_dict()
     step_ms = float(parts.sum(axis=1).mean())
     if dist:
         t = torch.tensor([step_ms], dtype=torch.float64, device=dev)
@@ -230,7 +246,7 @@ def run_ours(args, rank, world, local_rank):
         w0_pin.copy_(torch.from_numpy(w_t0_np))
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        e = ctx.fda_round_host(w_pin[:, :d], w0_pin, xi_pin, ALL_STATE, F.FDA_VARIANT_SKETCH, eps, theta,
+        e = ctx.fda_round_host(w_pin[:, :d], w0_pin, None, SKETCH_STATE, F.FDA_VARIANT_SKETCH, eps, theta,
                                0, st_pin)           # result: states, estimate, new global model
         dt = time.perf_counter() - t0
         if it >= 2:
@@ -241,13 +257,14 @@ def run_ours(args, rank, world, local_rank):
         t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
-    h2d = 4 * (K * d + 2 * d)
+    h2d = 4 * (K * d + d)
     d2h = 4 * (d + K * slen) + 88
 
     out = None
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
-        algo_bytes = 4.0 * (K * d + 2 * d + K * slen)        # w, w_t0, xi read; states written
+        algo_bytes = 4.0 * (K * d + d + K * slen)            # w, w_t0 read; states written
+        lin_bytes = 4.0 * (K * d + 2 * d + K * slen)         # + xi
         achieved = algo_bytes / (ls_ms * 1e-3) / 1e9
         cpu = None
         if world == 1 and not args.skip_cpu_baseline:
@@ -263,7 +280,7 @@ def run_ours(args, rank, world, local_rank):
             "data": "synthetic",
             "config": {"workload": "%d:%s d=%d K=%d sketch=%dx%d eps=%.4f theta=%g" %
                                    (args.workload, wl.name, d, K, wl.l, wl.m, wl.epsilon, theta),
-                       "state": "norm+projection+sketch", "variant": "sketch", "average": "broadcast in place",
+                       "state": "SketchFDA: norm+sketch", "variant": "sketch", "average": "broadcast in place",
                        "l2": "inputs (%.1f GB) larger than L2; models restored from a pristine copy before "
                              "each step, outside the timed events" % (4 * K * d / 1e9),
                        "multi_gpu": "replicas only"},
@@ -271,6 +288,9 @@ def run_ours(args, rank, world, local_rank):
             "local_state_only": {"value": K * d / (ls_ms * 1e-3), "unit": UNIT},
             "average_only": {"gbs": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9,
                              "frac_of_peak": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9 / peak},
+            "linear_local_state": {"ms": lin_ms, "value": K * d / (lin_ms * 1e-3), "unit": UNIT,
+                                   "gbs": lin_bytes / (lin_ms * 1e-3) / 1e9,
+                                   "frac_of_peak": lin_bytes / (lin_ms * 1e-3) / 1e9 / peak, "H": lin_est["H"]},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
             "roofline": {"kernel": "k_local_state", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,

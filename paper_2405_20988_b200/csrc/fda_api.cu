@@ -105,7 +105,8 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
         if (e == cudaSuccess)
             e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
     }
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * (size_t)ctx->max_blocks * 32 * 2);
+    ctx->part_np_doubles = (size_t)ctx->max_blocks * (size_t)(K_max > 32 ? K_max : 32) * 2;
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * ctx->part_np_doubles);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->err_flag, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(ctx->err_flag, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);

@@ -27,6 +27,7 @@ struct fda_ctx {
     float *part_sk = nullptr;         // per-block sketch partials
     size_t part_sk_floats = 0;
     double *part_np = nullptr;        // per-block (norm, projection) partials
+    size_t part_np_doubles = 0;
     int max_blocks = 0;
     unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
     // staging for fda_round_host (lazy)
@@ -45,6 +46,9 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s);
 cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, cudaStream_t s);
+cudaError_t fda_launch_local_state_linear(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);
 cudaError_t fda_setup_local_state(fda_ctx *ctx);   // opt-in shared memory, pick geometry

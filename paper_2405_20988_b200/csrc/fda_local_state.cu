@@ -467,6 +467,8 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
     {   // aligned sketch requests take the bulk-copy staged kernel
         cudaError_t e = fda_launch_local_state_staged(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
         if (e != cudaErrorNotSupported) return e;
+        e = fda_launch_local_state_linear(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
+        if (e != cudaErrorNotSupported) return e;
     }
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     LsParams p{};

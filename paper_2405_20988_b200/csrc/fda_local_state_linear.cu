@@ -1,0 +1,165 @@
+// Local-state pass without the sketch: ||u^(k)||^2 and <xi,u^(k)> only (Section 3, local
+// state; Section 3.2, LinearFDA).  Pure streaming: K*d + 2*d floats are read once.
+//
+// A block walks index tiles; w_t0 and xi of a tile are parked in shared memory once and every
+// warp then streams the rows of "its" workers (k = warp, warp + NW, ...) with coalesced
+// 128-bit loads, several in flight per lane.  fp32 partial sums cover one tile (at most 64
+// elements per lane), the running sums are fp64; each block writes one partial per worker and
+// a small second kernel adds the partials in block order.
+#include "fda_internal.h"
+
+namespace {
+
+constexpr int kTile = 2048;           // indices per tile
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunks = kTile / 128;  // 128 indices = one float4 per lane
+
+template <int KPW, bool LINEAR, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int64_t d,
+                     const float *__restrict__ w_t0, const float *__restrict__ xi, int64_t tiles,
+                     double *__restrict__ part_np /* [block][K][2] */)
+{
+    __shared__ __align__(16) float w0s[kTile];
+    __shared__ __align__(16) float xis[LINEAR ? kTile : 4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double acc_n[KPW], acc_p[KPW];
+#pragma unroll
+    for (int kk = 0; kk < KPW; ++kk) { acc_n[kk] = 0.0; acc_p[kk] = 0.0; }
+
+    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const int64_t j0 = tile * kTile;
+        __syncthreads();                                   // the previous tile is no longer read
+        for (int i = tid * 4; i < kTile; i += kThreads * 4) {
+            const int64_t j = j0 + i;
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f), x = b;
+            if (VEC && j + 3 < d) {
+                b = __ldg(reinterpret_cast<const float4 *>(w_t0 + j));
+                if (LINEAR) x = __ldg(reinterpret_cast<const float4 *>(xi + j));
+            } else {
+                if (j + 0 < d) { b.x = __ldg(w_t0 + j + 0); if (LINEAR) x.x = __ldg(xi + j + 0); }
+                if (j + 1 < d) { b.y = __ldg(w_t0 + j + 1); if (LINEAR) x.y = __ldg(xi + j + 1); }
+                if (j + 2 < d) { b.z = __ldg(w_t0 + j + 2); if (LINEAR) x.z = __ldg(xi + j + 2); }
+                if (j + 3 < d) { b.w = __ldg(w_t0 + j + 3); if (LINEAR) x.w = __ldg(xi + j + 3); }
+            }
+            *reinterpret_cast<float4 *>(w0s + i) = b;
+            if (LINEAR) *reinterpret_cast<float4 *>(xis + i) = x;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < KPW; ++kk) {
+            const int k = warp + kk * kWarps;
+            if (k >= K) continue;
+            const float *__restrict__ wk = w + (size_t)k * (size_t)row_stride;
+            float pn = 0.f, pp = 0.f;
+            constexpr int B = VEC ? 8 : 2;                 // row loads in flight per lane
+#pragma unroll 1
+            for (int c0 = 0; c0 < kChunks; c0 += B) {
+                float4 a[B];
+#pragma unroll
+                for (int c = 0; c < B; ++c) {
+                    const int64_t j = j0 + (c0 + c) * 128 + lane * 4;
+                    if (VEC && j + 3 < d) {
+                        a[c] = __ldcs(reinterpret_cast<const float4 *>(wk + j));
+                    } else {
+                        // past the end u must be 0: w_t0 is 0 there, so load 0 for w as well
+                        a[c].x = j + 0 < d ? __ldg(wk + j + 0) : 0.f;
+                        a[c].y = j + 1 < d ? __ldg(wk + j + 1) : 0.f;
+                        a[c].z = j + 2 < d ? __ldg(wk + j + 2) : 0.f;
+                        a[c].w = j + 3 < d ? __ldg(wk + j + 3) : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < B; ++c) {
+                    const int i = (c0 + c) * 128 + lane * 4;
+                    const float4 b = *reinterpret_cast<const float4 *>(w0s + i);
+                    const float ux = a[c].x - b.x, uy = a[c].y - b.y, uz = a[c].z - b.z, uw = a[c].w - b.w;
+                    pn = fmaf(ux, ux, pn); pn = fmaf(uy, uy, pn); pn = fmaf(uz, uz, pn); pn = fmaf(uw, uw, pn);
+                    if (LINEAR) {
+                        const float4 x = *reinterpret_cast<const float4 *>(xis + i);
+                        pp = fmaf(x.x, ux, pp); pp = fmaf(x.y, uy, pp); pp = fmaf(x.z, uz, pp); pp = fmaf(x.w, uw, pp);
+                    }
+                }
+            }
+            acc_n[kk] += (double)pn;
+            if (LINEAR) acc_p[kk] += (double)pp;
+        }
+    }
+#pragma unroll
+    for (int kk = 0; kk < KPW; ++kk) {
+        double n = acc_n[kk], pr = acc_p[kk];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            n += __shfl_xor_sync(0xffffffffu, n, off);
+            pr += __shfl_xor_sync(0xffffffffu, pr, off);
+        }
+        const int k = warp + kk * kWarps;
+        if (lane == 0 && k < K) {
+            part_np[((size_t)blockIdx.x * K + k) * 2 + 0] = n;
+            part_np[((size_t)blockIdx.x * K + k) * 2 + 1] = pr;
+        }
+    }
+}
+
+// states[k][0..1] = sum over blocks (block order, fp64); every sketch slot is written as 0.
+__global__ void k_finalize_linear(const double *__restrict__ part_np, int K, int blocks, int slen,
+                                  uint32_t flags, bool have_xi, float *__restrict__ states)
+{
+    const int64_t total = (int64_t)K * slen;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        const int k = (int)(t / slen), e = (int)(t % slen);
+        double acc = 0.0;
+        const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0
+                      : (e == 1) ? ((flags & FDA_STATE_LINEAR) != 0 && have_xi) : false;
+        if (on)
+            for (int b = 0; b < blocks; ++b) acc += part_np[((size_t)b * K + k) * 2 + e];
+        states[t] = (float)acc;
+    }
+}
+
+template <int KPW>
+cudaError_t launch_kpw(int blocks, bool linear, bool vec, const float *w, int64_t row_stride, int K, int64_t d,
+                       const float *w_t0, const float *xi, int64_t tiles, double *part, cudaStream_t s)
+{
+#define FDA_LIN(LI, VE) k_local_state_linear<KPW, LI, VE><<<blocks, kThreads, 0, s>>>(w, row_stride, K, d, w_t0, xi, tiles, part)
+    if (linear) { if (vec) FDA_LIN(true, true); else FDA_LIN(true, false); }
+    else        { if (vec) FDA_LIN(false, true); else FDA_LIN(false, false); }
+#undef FDA_LIN
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Returns cudaErrorNotSupported for requests this kernel does not take (sketch asked for, or
+// more workers than 8 per warp).
+cudaError_t fda_launch_local_state_linear(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, cudaStream_t s)
+{
+    if (flags & FDA_STATE_SKETCH) return cudaErrorNotSupported;
+    if (K > kWarps * 8) return cudaErrorNotSupported;
+    const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
+    const bool vec = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) &&
+                     (row_stride % 4 == 0);
+    const int64_t tiles = (d + kTile - 1) / kTile;
+    int64_t blocks = (int64_t)ctx->n_sm * 3;
+    if (blocks > tiles) blocks = tiles;
+    if (blocks > ctx->max_blocks) blocks = ctx->max_blocks;
+    if ((size_t)blocks * K * 2 > ctx->part_np_doubles) return cudaErrorNotSupported;
+    const int kpw = (K + kWarps - 1) / kWarps;
+    const bool linear = xi_used != nullptr;
+    cudaError_t e;
+    if (kpw <= 1)      e = launch_kpw<1>((int)blocks, linear, vec, w, row_stride, K, d, w_t0, xi_used, tiles, ctx->part_np, s);
+    else if (kpw <= 2) e = launch_kpw<2>((int)blocks, linear, vec, w, row_stride, K, d, w_t0, xi_used, tiles, ctx->part_np, s);
+    else if (kpw <= 4) e = launch_kpw<4>((int)blocks, linear, vec, w, row_stride, K, d, w_t0, xi_used, tiles, ctx->part_np, s);
+    else               e = launch_kpw<8>((int)blocks, linear, vec, w, row_stride, K, d, w_t0, xi_used, tiles, ctx->part_np, s);
+    if (e != cudaSuccess) return e;
+    const int slen = 2 + ctx->lm;
+    const int64_t total = (int64_t)K * slen;
+    int fb = (int)((total + 255) / 256);
+    if (fb > ctx->n_sm * 8) fb = ctx->n_sm * 8;
+    k_finalize_linear<<<fb, 256, 0, s>>>(ctx->part_np, K, (int)blocks, slen, flags, linear, states);
+    return cudaGetLastError();
+}
