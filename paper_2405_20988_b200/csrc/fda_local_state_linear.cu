@@ -3,7 +3,8 @@
 //
 // A block walks index tiles; w_t0 and xi of a tile are parked in shared memory once and every
 // warp then streams the rows of "its" workers (k = warp, warp + NW, ...) with coalesced
-// 128-bit loads, several in flight per lane.  fp32 partial sums cover one tile (at most 64
+// 128-bit loads, several in flight per lane.  With fewer workers than warps, several warps
+// share a worker and split the tile's chunks between them.  fp32 partial sums cover one tile (at most 64
 // elements per lane), the running sums are fp64; each block writes one partial per worker and
 // a small second kernel adds the partials in block order.
 #include "fda_internal.h"
@@ -24,6 +25,11 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
     __shared__ __align__(16) float w0s[kTile];
     __shared__ __align__(16) float xis[LINEAR ? kTile : 4];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // K < kWarps: warp -> (worker warp % K, share warp / K of nsub); otherwise one warp per worker slot
+    const int kc = K < kWarps ? K : kWarps;
+    const int nsub = kWarps / kc;
+    const int wslot = warp % kc, sub = warp / kc;
+    const bool idle = sub >= nsub;
     double acc_n[KPW], acc_p[KPW];
 #pragma unroll
     for (int kk = 0; kk < KPW; ++kk) { acc_n[kk] = 0.0; acc_p[kk] = 0.0; }
@@ -49,13 +55,13 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
         __syncthreads();
 #pragma unroll
         for (int kk = 0; kk < KPW; ++kk) {
-            const int k = warp + kk * kWarps;
-            if (k >= K) continue;
+            const int k = wslot + kk * kWarps;
+            if (k >= K || idle) continue;
             const float *__restrict__ wk = w + (size_t)k * (size_t)row_stride;
             float pn = 0.f, pp = 0.f;
             constexpr int B = VEC ? 8 : 2;                 // row loads in flight per lane
 #pragma unroll 1
-            for (int c0 = 0; c0 < kChunks; c0 += B) {
+            for (int c0 = sub * B; c0 < kChunks; c0 += B * nsub) {
                 float4 a[B];
 #pragma unroll
                 for (int c = 0; c < B; ++c) {
@@ -94,10 +100,17 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
             n += __shfl_xor_sync(0xffffffffu, n, off);
             pr += __shfl_xor_sync(0xffffffffu, pr, off);
         }
-        const int k = warp + kk * kWarps;
-        if (lane == 0 && k < K) {
-            part_np[((size_t)blockIdx.x * K + k) * 2 + 0] = n;
-            part_np[((size_t)blockIdx.x * K + k) * 2 + 1] = pr;
+        // warps that share a worker add up through shared memory (fixed order)
+        __syncthreads();
+        double *red = reinterpret_cast<double *>(w0s);           // [kWarps][2]
+        if (lane == 0) { red[warp * 2] = n; red[warp * 2 + 1] = pr; }
+        __syncthreads();
+        const int k = wslot + kk * kWarps;
+        if (lane == 0 && sub == 0 && k < K) {
+            double tn = 0.0, tp = 0.0;
+            for (int q = 0; q < nsub; ++q) { tn += red[(wslot + q * kc) * 2]; tp += red[(wslot + q * kc) * 2 + 1]; }
+            part_np[((size_t)blockIdx.x * K + k) * 2 + 0] = tn;
+            part_np[((size_t)blockIdx.x * K + k) * 2 + 1] = tp;
         }
     }
 }
