@@ -173,6 +173,39 @@ fda_status fda_round_host(fda_ctx *ctx, float *w_host, int64_t row_stride, int K
 fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets,
                           int8_t *signs, void *stream);
 
+/*
+ * Local state without a context and without any allocation.  (The paper has no counterpart
+ * to this call; it exists for the way some programs have to use the library.)
+ *
+ * Every other entry point works on an fda_ctx, and creating one calls cudaMalloc.  Some
+ * callers cannot do that: a monitoring hook that runs inside a training step while the
+ * framework's caching allocator owns all free device memory (a cudaMalloc there fails, or
+ * stalls the whole device while it is served), and embedders whose device-memory budget is
+ * fixed when the library is loaded.  For them this call computes, for each of the K rows of
+ * w, states[k][0] = ||w^(k) - w_t0||^2 and states[k][1] = <xi, w^(k) - w_t0> (the LinearFDA
+ * local state, Section 3.2 of the FDA paper), using as scratch a fixed array that is part of
+ * the library image: 1 MiB of device memory on every GPU that loads the library, held until
+ * the process exits.
+ *   device      CUDA device that owns the pointers
+ *   w, w_t0, xi as in fda_local_state (any alignment; xi may be NULL)
+ *   flags       FDA_STATE_NORM and/or FDA_STATE_LINEAR; slots not asked for are written as 0
+ *   states      out, K x 2 floats (not K x state_len)
+ * Limits: K <= FDA_NOALLOC_MAX_WORKERS, otherwise FDA_ERR_UNSUPPORTED and nothing is
+ * launched.  Neither this call nor anything it uses calls cudaMalloc, cudaFree or an
+ * allocating library routine.  The first call on a device looks up the device address of the
+ * scratch array (cudaGetSymbolAddress); make that first call before starting any stream
+ * capture.  All calls on a device share the one scratch array: two calls whose kernels
+ * overlap on the GPU (different streams, or different host threads) race on it and give
+ * wrong sums, so serialise them.  Nothing in the array has to be cleared between calls:
+ * every slot a call reads is first written by that call.
+ * Errors: INVALID_ARG (NULL w, w_t0 or states, K < 1, d < 1, row_stride < d, unknown flag,
+ * FDA_STATE_SKETCH, device out of range), UNSUPPORTED (K too large), CUDA.
+ */
+#define FDA_NOALLOC_MAX_WORKERS 64
+fda_status fda_local_state_linear_noalloc(int device, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

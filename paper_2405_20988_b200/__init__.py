@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     Estimate,
     FdaContext,
     FdaError,
+    fda_local_state_linear_noalloc,
+    FDA_NOALLOC_MAX_WORKERS,
     library_path,
     load_library,
 )

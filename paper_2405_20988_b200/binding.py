@@ -21,7 +21,9 @@ _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "
            4: "FDA_ERR_NOMEM"}
 
 EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state",
-           "fda_combine_estimate", "fda_average_models", "fda_round_host", "fda_debug_hash")
+           "fda_combine_estimate", "fda_average_models", "fda_round_host", "fda_debug_hash",
+           "fda_local_state_linear_noalloc")
+FDA_NOALLOC_MAX_WORKERS = 64
 
 
 class FdaError(RuntimeError):
@@ -71,6 +73,8 @@ def load_library():
     lib.fda_average_models.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp]
     lib.fda_round_host.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, c_int, f32, f32, u32, vp, vp, vp]
     lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
+    lib.fda_local_state_linear_noalloc.argtypes = [c_int, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
+    lib.fda_local_state_linear_noalloc.restype = c_int
     for name in ("fda_create", "fda_destroy", "fda_local_state", "fda_combine_estimate",
                  "fda_average_models", "fda_round_host", "fda_debug_hash"):
         getattr(lib, name).restype = c_int
@@ -102,6 +106,29 @@ def _rows(w, name="w"):
     K, d = w.shape
     stride = w.stride(0) if K > 1 else max(w.stride(0), d)
     return stride, K, d
+
+
+def fda_local_state_linear_noalloc(w, w_t0, xi, flags: int, states, stream=None):
+    """states[K, 2] <- (||u_k||^2, <xi,u_k>) of the K rows of ``w`` without a context.
+
+    For code that must not allocate device memory when it runs (for instance a hook inside a
+    training step, where the framework's allocator already holds all free memory): the C
+    entry point of the same name keeps its scratch in a fixed array inside the library and
+    this wrapper creates no tensor either - ``states`` is supplied by the caller.  K may not
+    exceed FDA_NOALLOC_MAX_WORKERS.  Calls that overlap on the device race on that scratch.
+    """
+    import torch
+    lib = load_library()
+    stride, K, d = _rows(w)
+    if states.dim() != 2 or states.shape[0] != K or states.shape[1] != 2 or not states.is_contiguous():
+        raise ValueError("states must be a contiguous K x 2 tensor")
+    st = lib.fda_local_state_linear_noalloc(w.device.index or 0, _dev_ptr(w, torch.float32, "w"), stride, K, d,
+                                            _dev_ptr(w_t0, torch.float32, "w_t0"),
+                                            _dev_ptr(xi, torch.float32, "xi"), flags,
+                                            _dev_ptr(states, torch.float32, "states"), _stream_ptr(stream))
+    if st != 0:
+        raise FdaError(st, "fda_local_state_linear_noalloc",
+                       "K exceeds FDA_NOALLOC_MAX_WORKERS" if st == 2 else "")
 
 
 class FdaContext:
