@@ -118,6 +118,20 @@ def clocks_rejected(c) -> bool:
     return bool(bad) or bool(stuck)
 
 
+# ------------------------------------------------------------------- multi-rank plumbing
+def max_over_ranks(value: float, dist, device="cpu") -> float:
+    """Slowest rank's time: every multi-GPU number is the max over ranks."""
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, units_per_rank: float, step_seconds: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling)."""
+    return world * units_per_rank / step_seconds
+
+
 # ----------------------------------------------------------------------- CPU baseline
 def oracle_step_on_sample(wl, w_host, w_t0, xi, coeffs, d_sample, threads):
     """One whole step of the CPU oracle on the first d_sample indices of every worker."""
@@ -232,9 +246,7 @@ def run_ours(args, rank, world, local_rank):
     lin_est = ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_LINEAR, eps, theta, est_buf).as_dict()
     step_ms = float(parts.sum(axis=1).mean())
     if dist:
-        t = torch.tensor([step_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms = float(t.item())
+        step_ms = max_over_ranks(step_ms, dist, dev)
     ls_ms, cb_ms, av_ms = (float(x) for x in parts.mean(axis=0))
 
     # ---- end to end through the host entry point (pinned buffers, copies timed) ----------
@@ -254,9 +266,7 @@ def run_ours(args, rank, world, local_rank):
         assert e.trigger == 1
     e2e_s = float(np.mean(e2e_times)) if e2e_times else float('nan')
     if dist:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, dist, dev)
     h2d = 4 * (K * d + d)
     d2h = 4 * (d + K * slen) + 88
 
@@ -274,7 +284,7 @@ def run_ours(args, rank, world, local_rank):
             cpu = {"value": K * d_s / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
                    "sample": "all %d workers x first %d of %d indices, one whole step, %.1f s" % (K, d_s, d, dt)}
         out = {
-            "metric": METRIC, "value": world * K * d / (step_ms * 1e-3), "unit": UNIT,
+            "metric": METRIC, "value": job_value(world, K * d, step_ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
@@ -298,7 +308,7 @@ def run_ours(args, rank, world, local_rank):
                          "traffic": LOCAL_STATE_TRAFFIC_BYTES.get(args.workload)},
             "cpu_baseline": cpu,
             "e2e": None if not e2e_times else
-                   {"value": world * K * d / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                   {"value": job_value(world, K * d, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "api": "fda_round_host"},
             "gpu_launches": 4 * args.steps,
             "clocks": clocks,

@@ -117,6 +117,19 @@ fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int
                            void *stream);
 
 /*
+ * Averaged state S-bar in one pass, without the K per-worker states: mean_state (one row of
+ * state_len floats) = ( (1/K) sum_k ||u^(k)||^2, (1/K) sum_k <xi,u^(k)>, sk(u-bar) ) with
+ * u-bar = (1/K) sum_k u^(k).  By the linearity of the sketch (Section 3.1, property (a); the
+ * "(lin.)" step in the proof of Theorem 1) sk(u-bar) equals the average of the K worker
+ * sketches that Algorithm 1 line 7 forms, so fda_combine_estimate(ctx, mean_state, K = 1, ...)
+ * yields the same H and trigger as the per-worker route, with l instead of K*l bin updates
+ * per index.  Arguments and errors as fda_local_state; mean_state is state_len floats.
+ */
+fda_status fda_mean_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
+                          const float *w_t0, const float *xi, uint32_t flags, float *mean_state,
+                          void *stream);
+
+/*
  * Average the K states and evaluate the variance over-estimate (Algorithm 1 lines 7-8).
  *   FDA_VARIANT_SKETCH: H = S-bar[0] - median_i ||row_i(S-bar sketch)||^2 / (1 + epsilon)
  *                       (Theorem 1; the median of an even number of rows is the mean of

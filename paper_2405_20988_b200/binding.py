@@ -20,7 +20,7 @@ FDA_MAX_ROWS = 16
 _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "FDA_ERR_CUDA",
            4: "FDA_ERR_NOMEM"}
 
-EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state",
+EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
            "fda_combine_estimate", "fda_average_models", "fda_round_host", "fda_debug_hash",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
@@ -69,6 +69,8 @@ def load_library():
     lib.fda_last_error.argtypes = [vp]
     lib.fda_last_error.restype = ctypes.c_char_p
     lib.fda_local_state.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
+    lib.fda_mean_state.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
+    lib.fda_mean_state.restype = c_int
     lib.fda_combine_estimate.argtypes = [vp, vp, c_int, c_int, f32, f32, vp, vp, vp]
     lib.fda_average_models.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp]
     lib.fda_round_host.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, c_int, f32, f32, u32, vp, vp, vp]
@@ -189,6 +191,16 @@ class FdaContext:
                                        _dev_ptr(xi, torch.float32, "xi"), flags,
                                        _dev_ptr(states, torch.float32, "states"), _stream_ptr(stream))
         self._check(st, "fda_local_state")
+
+    def fda_mean_state(self, w, w_t0, xi, flags: int, mean_state, stream=None):
+        """mean_state[state_len] <- averaged state S-bar of the K rows of w (device tensors)."""
+        import torch
+        stride, K, d = _rows(w)
+        st = self._lib.fda_mean_state(self._h, _dev_ptr(w, torch.float32, "w"), stride, K, d,
+                                      _dev_ptr(w_t0, torch.float32, "w_t0"),
+                                      _dev_ptr(xi, torch.float32, "xi"), flags,
+                                      _dev_ptr(mean_state, torch.float32, "mean_state"), _stream_ptr(stream))
+        self._check(st, "fda_mean_state")
 
     def fda_combine_estimate(self, states, K: int, variant: int, epsilon: float, theta: float,
                              est_dev, want_host: bool = True, stream=None):

@@ -42,6 +42,7 @@ void free_device(fda_ctx *ctx)
 {
     cudaFree(ctx->coeffs_dev);
     cudaFree(ctx->tab);
+    cudaFree(ctx->tab32);
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
     cudaFree(ctx->err_flag);
@@ -101,6 +102,8 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
+        if (e == cudaSuccess && (size_t)ctx->lm * 128 < ((size_t)1 << 31))
+            e = cudaMalloc(&ctx->tab32, sizeof(uint32_t) * (size_t)l * ctx->tab_stride);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
         if (e == cudaSuccess)
             e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
@@ -154,6 +157,27 @@ fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int
     cudaError_t e = fda_launch_local_state(ctx, w, row_stride, K, d, w_t0, xi, flags, states,
                                            (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_local_state");
+    return FDA_OK;
+}
+
+fda_status fda_mean_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
+                          const float *w_t0, const float *xi, uint32_t flags, float *mean_state,
+                          void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!w || !w_t0 || !mean_state) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: null pointer");
+    if (K < 1 || K > ctx->K_max) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: K out of range");
+    if (d < 1 || d > ctx->d_max) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: d out of range");
+    if (row_stride < d) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: row_stride < d");
+    if (flags & ~(uint32_t)(FDA_STATE_NORM | FDA_STATE_LINEAR | FDA_STATE_SKETCH))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: unknown flag");
+    if ((flags & FDA_STATE_SKETCH) && ctx->l == 0)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_mean_state: context has no sketch");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_mean_state: cannot select device");
+    cudaError_t e = fda_launch_mean_state(ctx, w, row_stride, K, d, w_t0, xi, flags, mean_state,
+                                          (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_mean_state");
     return FDA_OK;
 }
 

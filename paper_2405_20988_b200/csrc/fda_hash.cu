@@ -20,6 +20,23 @@ __global__ void k_build_table(const uint64_t *__restrict__ coeffs, int l, uint32
     (void)l;
 }
 
+// 32-bit variant for the staged sketch kernel: bits 0..30 hold the byte offset of the cell in a
+// bins[cell][32] float array, (i*m + bucket) * 128, bit 31 is set when the sign is -1, so that
+// the kernel needs one AND for the address and one AND-XOR for the signed value.
+__global__ void k_build_table32(const uint64_t *__restrict__ coeffs, uint32_t m, uint64_t magic, int64_t n,
+                                int64_t tab_stride, uint32_t *__restrict__ tab)
+{
+    const int i = blockIdx.y;
+    const uint64_t c[6] = {coeffs[6 * i + 0], coeffs[6 * i + 1], coeffs[6 * i + 2],
+                           coeffs[6 * i + 3], coeffs[6 * i + 4], coeffs[6 * i + 5]};
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n;
+         j += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t b = fda::bucket_of(c, (uint32_t)j, m, magic);
+        const uint32_t s = fda::sign_is_negative(c, (uint32_t)j) ? 0x80000000u : 0u;
+        tab[(size_t)i * tab_stride + j] = (((uint32_t)i * m + b) << 7) | s;
+    }
+}
+
 __global__ void k_debug_hash(const uint64_t *__restrict__ coeffs, uint32_t m, uint64_t magic,
                              int64_t j0, int64_t n, uint16_t *__restrict__ buckets,
                              int8_t *__restrict__ signs)
@@ -52,6 +69,9 @@ cudaError_t fda_launch_build_table(const fda_ctx *ctx, cudaStream_t s)
     dim3 grid(blocks_for(ctx->tab_stride, 256, ctx->n_sm * 16), (unsigned)ctx->l);
     k_build_table<<<grid, 256, 0, s>>>(ctx->coeffs_dev, ctx->l, (uint32_t)ctx->m, magic,
                                       ctx->tab_stride, ctx->tab_stride, ctx->tab);
+    if (ctx->tab32)
+        k_build_table32<<<grid, 256, 0, s>>>(ctx->coeffs_dev, (uint32_t)ctx->m, magic, ctx->tab_stride,
+                                            ctx->tab_stride, ctx->tab32);
     return cudaGetLastError();
 }
 

@@ -23,6 +23,7 @@ struct fda_ctx {
     // device scratch
     uint64_t *coeffs_dev = nullptr;   // 6*l
     uint16_t *tab = nullptr;          // l planes of tab_stride entries
+    uint32_t *tab32 = nullptr;        // same hash as byte offset | sign<<31 (staged sketch kernel)
     int64_t tab_stride = 0;
     float *part_sk = nullptr;         // per-block sketch partials
     size_t part_sk_floats = 0;
@@ -51,6 +52,9 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
 cudaError_t fda_launch_local_state_linear(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);
+cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
+                                  const float *w_t0, const float *xi, uint32_t flags, float *mean_state,
+                                  cudaStream_t s);
 cudaError_t fda_setup_local_state(fda_ctx *ctx);   // opt-in shared memory, pick geometry
 cudaError_t fda_launch_combine(const fda_ctx *ctx, const float *states, int K, int variant,
                                float epsilon, float theta, fda_estimate *est_dev, cudaStream_t s);

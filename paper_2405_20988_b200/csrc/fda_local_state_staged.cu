@@ -125,7 +125,7 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 //        W  [Kg][bx] floats        at b*wbox_bytes
 //        W0 [bx] floats            at nb*wbox_bytes + b*vbox_bytes
 //        XI [bx] floats            at nb*(wbox_bytes + vbox_bytes) + b*vbox_bytes
-//        H  [rows_per_role][bx+4] uint16  at nb*(wbox_bytes + 2*vbox_bytes) + b*hbox_bytes
+//        H  [rows_per_role][bx] uint32    at nb*(wbox_bytes + 2*vbox_bytes) + b*hbox_bytes
 template <int LWK, bool LINEAR>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap tm_w,
@@ -156,7 +156,7 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
     const uint32_t bins_addr = smem_base + 128;
     const int local_cells = p.rows_per_role * p.m;
     const uint32_t bins_bytes = (uint32_t)local_cells * 32u * 4u;
-    const int S = p.stages, nb = p.nb, bx = p.bx, hbx = p.bx + 4;
+    const int S = p.stages, nb = p.nb, bx = p.bx;
     const uint32_t w0_off = (uint32_t)nb * p.wbox_bytes;
     const uint32_t xi_off = w0_off + (uint32_t)nb * p.vbox_bytes;
     const uint32_t h_off = xi_off + (uint32_t)nb * p.vbox_bytes;
@@ -178,11 +178,10 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
     const int64_t my_tiles = p.tiles > c ? (p.tiles - c + cpg - 1) / cpg : 0;
     // a tensor copy always delivers its whole box (zero-filled where outside the tensor)
     const uint32_t tx_bytes = (uint32_t)nb * ((uint32_t)(p.Kg * bx) * 4u + (uint32_t)bx * 4u * (LINEAR ? 2u : 1u) +
-                                              (uint32_t)(p.rows_per_role * hbx) * 2u);
+                                              (uint32_t)(p.rows_per_role * bx) * 4u);
 
     double acc_n = 0.0, acc_p = 0.0;
     const uint32_t col_addr = bins_addr + (uint32_t)lane * 4u;
-    const uint32_t row_bytes = (uint32_t)p.m * 128u;               // one sketch row of bins
     const int qpb = bx / 4;                                        // quads per box
     const int quads = qpb * nb;                                    // quads per tile
     const int quads_per_pass = ncons * JS * 2;
@@ -202,9 +201,7 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                 const bool in = q < quads;
                 any |= in;
                 const int b = in ? q / qpb : 0, xq = in ? q - b * qpb : 0;
-                // table box starts at the index rounded down to a multiple of 8
-                const uint32_t hskip = (uint32_t)((j0 + (int64_t)b * bx) & 7);
-                haddr[v] = base + h_off + (uint32_t)b * p.hbox_bytes + (hskip + 4u * (uint32_t)xq) * 2u;
+                haddr[v] = base + h_off + (uint32_t)b * p.hbox_bytes + 16u * (uint32_t)xq;
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), w0 = a;
                 if (in) {
                     a = lds_f32x4(base + (uint32_t)b * p.wbox_bytes + ((uint32_t)(kl * bx) + 4u * (uint32_t)xq) * 4u);
@@ -227,41 +224,43 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                 if (LINEAR) acc_p += (double)pp;
             }
             for (int i = 0; i < rows; ++i) {
-                uint32_t addr[NB];
+                uint32_t addr[NB], got[NB];
                 float val[NB], old[NB];
-                const uint32_t rowaddr = col_addr + (uint32_t)i * row_bytes;
 #pragma unroll
                 for (int v = 0; v < 2; ++v) {
-                    uint32_t hx, hy;        // 4 table entries of this quad (u = 0 where the quad is absent)
-                    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];"
-                                 : "=r"(hx), "=r"(hy) : "r"(haddr[v] + (uint32_t)(i * hbx) * 2u));
-                    addr[4 * v + 0] = rowaddr + ((hx & 0x7fffu) << 7);
-                    addr[4 * v + 1] = rowaddr + (((hx >> 16) & 0x7fffu) << 7);
-                    addr[4 * v + 2] = rowaddr + ((hy & 0x7fffu) << 7);
-                    addr[4 * v + 3] = rowaddr + (((hy >> 16) & 0x7fffu) << 7);
-                    val[4 * v + 0] = flip(u[4 * v + 0], (hx << 16) & 0x80000000u);
-                    val[4 * v + 1] = flip(u[4 * v + 1], hx & 0x80000000u);
-                    val[4 * v + 2] = flip(u[4 * v + 2], (hy << 16) & 0x80000000u);
-                    val[4 * v + 3] = flip(u[4 * v + 3], hy & 0x80000000u);
+                    // 4 table words of this quad: cell byte offset | sign << 31 (u = 0 where the quad is absent)
+                    uint32_t h[4];
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(haddr[v] + (uint32_t)(i * bx) * 4u));
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        addr[4 * v + e] = col_addr + (h[e] & 0x7fffffffu);
+                        val[4 * v + e] = flip(u[4 * v + e], h[e] & 0x80000000u);
+                    }
                 }
 #pragma unroll
                 for (int e = 0; e < NB; ++e) old[e] = lds_f32(addr[e]);
-                uint32_t lost = 0;          // bit e: the compare-and-swap of update e lost a race
+                uint32_t diff = 0;          // non-zero when some compare-and-swap of the eight lost a race
 #pragma unroll
                 for (int e = 0; e < NB; ++e) {
-                    const uint32_t got = cas_shared(addr[e], __float_as_uint(old[e]), __float_as_uint(old[e] + val[e]));
-                    lost |= (got != __float_as_uint(old[e])) ? (1u << e) : 0u;
+                    got[e] = cas_shared(addr[e], __float_as_uint(old[e]), __float_as_uint(old[e] + val[e]));
+                    diff |= got[e] ^ __float_as_uint(old[e]);
                 }
-                // redo the lost ones, one per lane and round, so that the lanes of a warp share
-                // the retry instruction whichever of their eight updates failed
-                while (lost) {
-                    uint32_t a = addr[0];
-                    float v = val[0];
+                if (diff) {
+                    // redo the lost ones, one per lane and round, so that the lanes of a warp share
+                    // the retry instruction whichever of their eight updates failed
+                    uint32_t lost = 0;
 #pragma unroll
-                    for (int e = 1; e < NB; ++e)
-                        if ((lost & ((1u << e) - 1u)) == 0 && (lost & (1u << e))) { a = addr[e]; v = val[e]; }
-                    red_shared_add(a, v);
-                    lost &= lost - 1u;
+                    for (int e = 0; e < NB; ++e) lost |= (got[e] != __float_as_uint(old[e])) ? (1u << e) : 0u;
+                    while (lost) {
+                        uint32_t a = addr[0];
+                        float v = val[0];
+#pragma unroll
+                        for (int e = 1; e < NB; ++e)
+                            if ((lost & ((1u << e) - 1u)) == 0 && (lost & (1u << e))) { a = addr[e]; v = val[e]; }
+                        red_shared_add(a, v);
+                        lost &= lost - 1u;
+                    }
                 }
             }
         }
@@ -292,7 +291,7 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                     tma_load_2d(base + (uint32_t)b * p.wbox_bytes, &tm_w, x, g * p.Kg, mbar);
                     tma_load_2d(base + w0_off + (uint32_t)b * p.vbox_bytes, &tm_w0, x, 0, mbar);
                     if (LINEAR) tma_load_2d(base + xi_off + (uint32_t)b * p.vbox_bytes, &tm_xi, x, 0, mbar);
-                    tma_load_2d(base + h_off + (uint32_t)b * p.hbox_bytes, &tm_tab, x & ~7, row0, mbar);
+                    tma_load_2d(base + h_off + (uint32_t)b * p.hbox_bytes, &tm_tab, x, row0, mbar);
                 }
             }
             __syncwarp();
@@ -449,7 +448,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s)
 {
-    if (!(flags & FDA_STATE_SKETCH) || ctx->l == 0) return cudaErrorNotSupported;
+    if (!(flags & FDA_STATE_SKETCH) || ctx->l == 0 || !ctx->tab32) return cudaErrorNotSupported;
     const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
     const bool aligned = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) &&
                          (row_stride % 4 == 0);
@@ -471,7 +470,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     const size_t row_bins = (size_t)ctx->m * 32 * sizeof(float);
     auto stage_size = [&](int rows, int bx, int nb) -> size_t {
         return (size_t)nb * (align128((size_t)p.Kg * bx * 4) + 2 * align128((size_t)bx * 4) +
-                             align128((size_t)rows * (bx + 4) * 2));
+                             align128((size_t)rows * bx * 4));
     };
     auto best_tile = [&](int rows, int stages, int *bx_out, int *nb_out) -> int {
         int best = 0;
@@ -502,7 +501,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     p.tiles = (d + tile - 1) / tile;
     p.wbox_bytes = (uint32_t)align128((size_t)p.Kg * bx * 4);
     p.vbox_bytes = (uint32_t)align128((size_t)bx * 4);
-    p.hbox_bytes = (uint32_t)align128((size_t)p.rows_per_role * (bx + 4) * 2);
+    p.hbox_bytes = (uint32_t)align128((size_t)p.rows_per_role * bx * 4);
     const int units = p.roles * p.groups;
     if (units > kMaxUnits || units > ctx->n_sm) return cudaErrorNotSupported;
 
@@ -544,9 +543,8 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     ok = ok && make_map(&maps[1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w_t0, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
     ok = ok && make_map(&maps[2], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, xi_used ? xi_used : w_t0, (uint64_t)d, 1,
                         vec_pitch, (uint32_t)bx, 1);
-    ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT16, ctx->tab, (uint64_t)ctx->tab_stride,
-                        (uint64_t)ctx->l, (uint64_t)ctx->tab_stride * 2, (uint32_t)(bx + 4),
-                        (uint32_t)p.rows_per_role);
+    ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT32, ctx->tab32, (uint64_t)ctx->tab_stride,
+                        (uint64_t)ctx->l, (uint64_t)ctx->tab_stride * 4, (uint32_t)bx, (uint32_t)p.rows_per_role);
     if (!ok) return cudaErrorNotSupported;
 
     size_t smem = 128 + (size_t)p.rows_per_role * row_bins + (size_t)p.stages * stage_size(p.rows_per_role, bx, nb);

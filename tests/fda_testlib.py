@@ -55,3 +55,21 @@ def check_average(gpu_avg, ora_avg, mean_abs=None):
     err = float(np.max(np.abs(g - o) / scale)) if o.size else 0.0
     assert err <= REL, err
     return err
+
+
+def check_mean_state(gpu_mean, ora_states, ubar_sq, l, m, d, K, sketch=True):
+    """Averaged state S-bar (fp32, one pass on the GPU) against the mean of the oracle's K
+    states.  Scales: the averaged projection and the cells of sk(u-bar) have the size of a
+    random projection / sketch cell of u-bar, so they are compared relative to
+    max(|value|, sqrt(||u-bar||^2/d)) and max(|cell|, sqrt(||u-bar||^2/m)); each of the K drifts
+    entering the sum carries its own fp32 rounding, hence the extra sqrt(K) allowance."""
+    g = np.asarray(gpu_mean, dtype=np.float64)
+    o = np.asarray(ora_states, dtype=np.float64).mean(axis=0)
+    assert abs(g[0] - o[0]) <= REL * o[0] + 1e-300
+    slack = np.sqrt(K)
+    pscale = max(abs(o[1]), np.sqrt(ubar_sq / d), 1e-300)
+    assert abs(g[1] - o[1]) <= REL * slack * pscale
+    if l > 0 and sketch:
+        scale = np.maximum(np.maximum(np.abs(o[2:]), np.sqrt(ubar_sq / m)), 1e-300)
+        err = float(np.max(np.abs(g[2:] - o[2:]) / scale))
+        assert err <= REL * slack, err

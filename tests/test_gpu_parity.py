@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 import fda_synth as S
-from fda_testlib import REL, check_average, check_estimate, check_states, check_trigger
+from fda_testlib import REL, check_average, check_estimate, check_mean_state, check_states, check_trigger
 
 pytestmark = pytest.mark.gpu
 
@@ -200,6 +200,50 @@ def test_heavy_tailed_values(env):
     check_states(got, ora, wl.l, wl.m, wl.d)
 
 
+# ------------------------------------------------------------------- averaged state
+@pytest.mark.parametrize("K,d,l,m,misalign", [
+    (1, 1, 5, 250, 0), (2, 7, 3, 7, 0), (5, 4099, 5, 250, 0), (8, 100_003, 5, 250, 0), (30, 20_001, 5, 250, 0),
+    (60, 30_011, 7, 500, 0), (9, 9_999, 16, 1000, 0), (13, 10_007, 5, 250, 3), (4, 3_000, 2, 20_000, 0),
+])
+def test_mean_state_matches_mean_of_oracle_states(env, K, d, l, m, misalign):
+    """sk(u-bar) = mean_k sk(u_k) (linearity, Section 3.1): the one-pass averaged state against
+    the average of the oracle's per-worker states, and the estimate it leads to."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(K * 7919 + d)
+    stride = S.row_stride(d) + (1 if misalign else 0)
+    coeffs = rand_coeffs(rng, l)
+    w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+    wbuf = np.zeros((K, stride), dtype=np.float32)
+    wbuf[:, :d] = w_t0 + (rng.normal(2e-4, 1e-3, size=(K, d))).astype(np.float32)
+    xi = rng.normal(size=d)
+    xi = (xi / np.linalg.norm(xi)).astype(np.float32)
+    ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, l, m, threads=4)
+    _, _, ubar_sq = oracle.variance(wbuf[:, :d], w_t0)
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        w, w0, xg, _ = gpu_states(torch, F, ctx, wbuf, w_t0, xi, ALL, misalign)
+        mean = torch.full((ctx.state_len,), float("nan"), dtype=torch.float32, device="cuda")
+        buf = ctx.new_estimate_buffer()
+        for flags in (ALL, 1 | 4, 1 | 2):
+            ctx.fda_mean_state(w[:, :d], w0, xg, flags, mean)
+            torch.cuda.synchronize()
+            got = mean.cpu().numpy()
+            ref = ora.copy()
+            if not flags & 2:
+                ref[:, 1] = 0
+            if not flags & 4:
+                assert not got[2:].any()
+            check_mean_state(got, ref, ubar_sq, l, m, d, K, sketch=bool(flags & 4))
+        ctx.fda_mean_state(w[:, :d], w0, xg, ALL, mean)
+        for variant in (0, 1):
+            e = ctx.fda_combine_estimate(mean.view(1, -1), 1, variant, 0.06, 1e-3, buf).as_dict()
+            r = oracle.combine(ora, l, m, variant, 0.06, 1e-3)
+            assert abs(e["mean_sq"] - r["mean_sq"]) <= REL * r["mean_sq"]
+            assert abs(e["est"] - r["est"]) <= 4 * REL * np.sqrt(K) * max(r["est"], ubar_sq)
+            tol = REL * r["mean_sq"] + 4 * REL * np.sqrt(K) * max(r["est"], ubar_sq)
+            assert abs(e["H"] - r["H"]) <= tol
+            check_trigger(e, r, 1e-3, tol)
+
+
 # ------------------------------------------------------------------- combine / trigger
 def test_combine_matches_oracle_on_gpu_states(env):
     torch, oracle, F = env
@@ -340,6 +384,20 @@ def full_round(env, idx, workers_for_oracle=None, check_avg_ranges=None):
                     ref2 = oracle.combine(ora, wl.l, wl.m, variant, wl.epsilon, float(np.float32(theta)))
                     tol2 = check_estimate(e, ref2, wl.l)
                     check_trigger(e, ref2, theta, tol2)
+        # the one-pass averaged state agrees with the average of the K states (linearity)
+        mean = torch.empty((ctx.state_len,), dtype=torch.float32, device="cuda")
+        ctx.fda_mean_state(w[:, :d], w0, xg, ALL, mean)
+        torch.cuda.synchronize()
+        gm, avg_states = mean.cpu().numpy().astype(np.float64), got.astype(np.float64).mean(axis=0)
+        ubar_sq = float(results[(F.FDA_VARIANT_SKETCH, wl.thetas[-1])]["est"]) * (1 + wl.epsilon)
+        assert abs(gm[0] - avg_states[0]) <= 2 * REL * avg_states[0]
+        cell_scale = np.maximum(np.abs(avg_states[2:]), np.sqrt(ubar_sq / wl.m))
+        assert np.max(np.abs(gm[2:] - avg_states[2:]) / cell_scale) <= 2 * REL * np.sqrt(K)
+        e_mean = ctx.fda_combine_estimate(mean.view(1, -1), 1, F.FDA_VARIANT_SKETCH, np.float32(wl.epsilon),
+                                          wl.thetas[-1], buf).as_dict()
+        e_ref = results[(F.FDA_VARIANT_SKETCH, wl.thetas[-1])]
+        assert abs(e_mean["H"] - e_ref["H"]) <= 8 * REL * np.sqrt(K) * (abs(e_ref["mean_sq"]) + abs(e_ref["est"]))
+        assert e_mean["trigger"] == e_ref["trigger"]
         # average (gated by the last sketch estimate, which fires on every workload)
         e = ctx.fda_combine_estimate(st, K, F.FDA_VARIANT_SKETCH, np.float32(wl.epsilon), wl.thetas[-1], buf)
         assert e.trigger == 1
