@@ -61,7 +61,7 @@ def host_cores() -> int:
 
 # ------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """nvidia-smi sampler (200 ms) running beside the timed region; read-only queries."""
+    """nvidia-smi sampler (100 ms) running beside the timed region; read-only queries."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
@@ -73,7 +73,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -244,6 +244,20 @@ def run_ours(args, rank, world, local_rank):
             lin_ms.append(e0.elapsed_time(e1))
     lin_ms = float(np.mean(lin_ms))
     lin_est = ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_LINEAR, eps, theta, est_buf).as_dict()
+
+    # ---- the one-pass averaged state (sketch of the mean drift, by linearity) ----
+    mean_state = torch.empty((ctx.state_len,), dtype=torch.float32, device=dev)
+    mean_ms = []
+    for it in range(3 + 10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.fda_mean_state(w[:, :d], w0, None, SKETCH_STATE, mean_state)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            mean_ms.append(e0.elapsed_time(e1))
+    mean_ms = float(np.mean(mean_ms))
+    mean_est = ctx.fda_combine_estimate(mean_state.view(1, -1), 1, F.FDA_VARIANT_SKETCH, eps, theta, est_buf).as_dict()
     step_ms = float(parts.sum(axis=1).mean())
     if dist:
         step_ms = max_over_ranks(step_ms, dist, dev)
@@ -301,6 +315,10 @@ def run_ours(args, rank, world, local_rank):
             "linear_local_state": {"ms": lin_ms, "value": K * d / (lin_ms * 1e-3), "unit": UNIT,
                                    "gbs": lin_bytes / (lin_ms * 1e-3) / 1e9,
                                    "frac_of_peak": lin_bytes / (lin_ms * 1e-3) / 1e9 / peak, "H": lin_est["H"]},
+            "mean_state": {"ms": mean_ms, "value": K * d / (mean_ms * 1e-3), "unit": UNIT,
+                           "gbs": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9,
+                           "frac_of_peak": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9 / peak,
+                           "H": mean_est["H"], "note": "fda_mean_state: S-bar in one pass, no per-worker sketches"},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
             "roofline": {"kernel": "k_local_state", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
@@ -355,7 +373,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", type=int, default=5, choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

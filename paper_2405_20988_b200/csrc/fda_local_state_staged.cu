@@ -459,8 +459,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     p.l = ctx->l; p.m = ctx->m;
     p.part_sk = ctx->part_sk; p.part_np = ctx->part_np; p.err_flag = ctx->err_flag;
 
-    int lwk = pow2_ceil(K < 32 ? K : 32);
-    if (lwk < 8) lwk = 8;
+    const int lwk = pow2_ceil(K < 32 ? K : 32);      // worker lanes per index slot
     p.groups = (K + lwk - 1) / lwk;
     p.Kg = (K + p.groups - 1) / p.groups;
 
@@ -552,6 +551,9 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     if (smem < smem_min) smem = smem_min;
     const bool linear = xi_used != nullptr;
     switch (lwk) {
+        case 1:  return launch<1>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
+        case 2:  return launch<2>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
+        case 4:  return launch<4>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
         case 8:  return launch<8>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
         case 16: return launch<16>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
         default: return launch<32>(ctx, p, maps, linear, blocks, threads, smem, flags, states, s);
