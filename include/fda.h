@@ -123,7 +123,9 @@ fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int
  * "(lin.)" step in the proof of Theorem 1) sk(u-bar) equals the average of the K worker
  * sketches that Algorithm 1 line 7 forms, so fda_combine_estimate(ctx, mean_state, K = 1, ...)
  * yields the same H and trigger as the per-worker route, with l instead of K*l bin updates
- * per index.  Arguments and errors as fda_local_state; mean_state is state_len floats.
+ * per index.  Arguments and errors as fda_local_state; mean_state is state_len floats.  The
+ * first call on a context allocates d_max floats of scratch for the average drift (NOMEM if
+ * that fails).
  */
 fda_status fda_mean_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                           const float *w_t0, const float *xi, uint32_t flags, float *mean_state,

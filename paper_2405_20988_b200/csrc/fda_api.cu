@@ -46,6 +46,7 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
     cudaFree(ctx->err_flag);
+    cudaFree(ctx->mean_model);
     cudaFree(ctx->stage_w);
     cudaFree(ctx->stage_w_t0);
     cudaFree(ctx->stage_xi);

@@ -30,6 +30,7 @@ struct fda_ctx {
     double *part_np = nullptr;        // per-block (norm, projection) partials
     size_t part_np_doubles = 0;
     int max_blocks = 0;
+    float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
     unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
     // staging for fda_round_host (lazy)
     float *stage_w = nullptr, *stage_w_t0 = nullptr, *stage_xi = nullptr, *stage_states = nullptr;
