@@ -163,6 +163,19 @@ fda_status fda_average_models(fda_ctx *ctx, float *w, int64_t row_stride, int K,
                               void *stream);
 
 /*
+ * fda_average_models that also refreshes the LinearFDA direction (Section 3.2, the heuristic
+ * choice of xi; Table 1): xi_out := (w-bar_new - w_t0_old) / ||w-bar_new - w_t0_old||, the
+ * normalised step of the global model between the last two synchronisations, computed in the
+ * same pass that averages (w_t0 is read before it is overwritten).  xi_out is d floats and is
+ * left untouched when the gate does not fire; it becomes all zero when the step is exactly
+ * zero.  xi_out must not alias w or w_t0.  Errors as fda_average_models, plus INVALID_ARG for
+ * a NULL xi_out.
+ */
+fda_status fda_average_models_xi(fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                                 float *w_t0, float *xi_out, const fda_estimate *est_dev,
+                                 uint32_t flags, void *stream);
+
+/*
  * One whole round on HOST buffers: copies w, w_t0 and xi to device staging owned by the
  * context (allocated on first use for K_max x d_max), runs fda_local_state,
  * fda_combine_estimate and fda_average_models (FDA_AVG_BROADCAST, gated by the trigger) and

@@ -14,5 +14,6 @@ from .fda_oracle import (  # noqa: F401
     combine,
     average,
     variance,
+    direction,
     state_len,
 )

@@ -35,6 +35,7 @@
 #include <stddef.h>
 #include <stdlib.h>
 #include <string.h>
+#include <math.h>
 
 typedef unsigned __int128 u128;
 
@@ -214,5 +215,22 @@ int fda_oracle_variance(const float *w, int64_t row_stride, int K, int64_t d,
     out[0] = var / (double)K;
     out[1] = msq / (double)K;
     out[2] = ubar2;
+    return 0;
+}
+
+/* LinearFDA direction heuristic (Section 3.2, Table 1): xi = (w_new - w_old) / ||w_new - w_old||,
+ * the normalised step of the global model between two synchronisations.  w_new is the fp64
+ * average model, w_old the fp32 model it replaces.  A zero step gives xi = 0. */
+int fda_oracle_direction(const double *w_new, const float *w_old, int64_t d, double *xi)
+{
+    if (!w_new || !w_old || !xi || d < 1) return 1;
+    double sq = 0.0;
+    for (int64_t j = 0; j < d; ++j) {
+        double dl = w_new[j] - (double)w_old[j];
+        sq += dl * dl;
+    }
+    double norm = sqrt(sq);
+    for (int64_t j = 0; j < d; ++j)
+        xi[j] = norm > 0.0 ? (w_new[j] - (double)w_old[j]) / norm : 0.0;
     return 0;
 }

@@ -48,6 +48,8 @@ def _load():
         lib.fda_oracle_combine.argtypes = [vp, c_int, c_int, c_int, c_int, c_dbl, c_dbl, vp]
         lib.fda_oracle_average.argtypes = [vp, c_i64, c_int, c_i64, c_i64, c_i64, vp]
         lib.fda_oracle_variance.argtypes = [vp, c_i64, c_int, c_i64, vp, vp]
+        lib.fda_oracle_direction.argtypes = [vp, vp, c_i64, vp]
+        lib.fda_oracle_direction.restype = c_int
         for f in (lib.fda_oracle_hash, lib.fda_oracle_local_state, lib.fda_oracle_combine,
                   lib.fda_oracle_average, lib.fda_oracle_variance):
             f.restype = c_int
@@ -167,3 +169,16 @@ def variance(w, w_t0):
     if rc:
         raise ValueError("fda_oracle_variance rejected its arguments")
     return float(out[0]), float(out[1]), float(out[2])
+
+
+def direction(w_new, w_old):
+    """Unit direction of the global step, (w_new - w_old)/||.||, in fp64 (zero step -> zeros)."""
+    w_new = np.ascontiguousarray(w_new, dtype=np.float64)
+    w_old = np.ascontiguousarray(w_old, dtype=np.float32)
+    if w_new.shape != w_old.shape or w_new.ndim != 1:
+        raise ValueError("w_new and w_old must be vectors of equal length")
+    out = np.empty_like(w_new)
+    rc = _load().fda_oracle_direction(_ptr(w_new), _ptr(w_old), w_new.size, _ptr(out))
+    if rc:
+        raise ValueError("fda_oracle_direction rejected its arguments")
+    return out

@@ -20,3 +20,4 @@ from .binding import (  # noqa: F401
     library_path,
     load_library,
 )
+from .rounds import run_rounds  # noqa: F401

@@ -21,7 +21,7 @@ _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "
            4: "FDA_ERR_NOMEM"}
 
 EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
-           "fda_combine_estimate", "fda_average_models", "fda_round_host", "fda_debug_hash",
+           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
 
@@ -73,6 +73,8 @@ def load_library():
     lib.fda_mean_state.restype = c_int
     lib.fda_combine_estimate.argtypes = [vp, vp, c_int, c_int, f32, f32, vp, vp, vp]
     lib.fda_average_models.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, vp]
+    lib.fda_average_models_xi.argtypes = [vp, vp, i64, c_int, i64, vp, vp, vp, u32, vp]
+    lib.fda_average_models_xi.restype = c_int
     lib.fda_round_host.argtypes = [vp, vp, i64, c_int, i64, vp, vp, u32, c_int, f32, f32, u32, vp, vp, vp]
     lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
     lib.fda_local_state_linear_noalloc.argtypes = [c_int, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
@@ -223,6 +225,17 @@ class FdaContext:
                                           _dev_ptr(est_dev, torch.uint8, "est_dev"), flags,
                                           _stream_ptr(stream))
         self._check(st, "fda_average_models")
+
+    def fda_average_models_xi(self, w, w_t0, xi_out, est_dev, flags: int, stream=None):
+        """fda_average_models that also writes the refreshed unit direction xi_out (d floats)."""
+        import torch
+        stride, K, d = _rows(w)
+        st = self._lib.fda_average_models_xi(self._h, _dev_ptr(w, torch.float32, "w"), stride, K, d,
+                                             _dev_ptr(w_t0, torch.float32, "w_t0"),
+                                             _dev_ptr(xi_out, torch.float32, "xi_out"),
+                                             _dev_ptr(est_dev, torch.uint8, "est_dev"), flags,
+                                             _stream_ptr(stream))
+        self._check(st, "fda_average_models_xi")
 
     def fda_round_host(self, w_host, w_t0_host, xi_host, state_flags: int, variant: int,
                        epsilon: float, theta: float, avg_flags: int, states_host=None, stream=None):

@@ -225,9 +225,27 @@ fda_status fda_average_models(fda_ctx *ctx, float *w, int64_t row_stride, int K,
         return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models: unknown flag");
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_average_models: cannot select device");
-    cudaError_t e = fda_launch_average(ctx, w, row_stride, K, d, w_t0, est_dev, flags,
+    cudaError_t e = fda_launch_average(ctx, w, row_stride, K, d, w_t0, nullptr, est_dev, flags,
                                        (cudaStream_t)stream);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_average_models");
+    return FDA_OK;
+}
+
+fda_status fda_average_models_xi(fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
+                                 float *w_t0, float *xi_out, const fda_estimate *est_dev,
+                                 uint32_t flags, void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!w || !w_t0 || !xi_out) return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models_xi: null pointer");
+    if (K < 1 || d < 1 || row_stride < d)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models_xi: size out of range");
+    if (flags & ~(uint32_t)(FDA_AVG_BROADCAST | FDA_AVG_UNCONDITIONAL))
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_average_models_xi: unknown flag");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_average_models_xi: cannot select device");
+    cudaError_t e = fda_launch_average(ctx, w, row_stride, K, d, w_t0, xi_out, est_dev, flags,
+                                       (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_average_models_xi");
     return FDA_OK;
 }
 

@@ -60,7 +60,7 @@ cudaError_t fda_setup_local_state(fda_ctx *ctx);   // opt-in shared memory, pick
 cudaError_t fda_launch_combine(const fda_ctx *ctx, const float *states, int K, int variant,
                                float epsilon, float theta, fda_estimate *est_dev, cudaStream_t s);
 cudaError_t fda_launch_average(const fda_ctx *ctx, float *w, int64_t row_stride, int K, int64_t d,
-                               float *w_t0, const fda_estimate *est_dev, uint32_t flags,
+                               float *w_t0, float *xi_out, const fda_estimate *est_dev, uint32_t flags,
                                cudaStream_t s);
 
 #endif

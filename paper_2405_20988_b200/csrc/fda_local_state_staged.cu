@@ -28,7 +28,9 @@
 // Updates.  Eight shared-memory updates per lane are in flight (eight loads, eight adds,
 // eight compare-and-swaps); an update whose compare-and-swap lost a race is redone with an
 // atomic add.  Lanes own their column, so races only occur between warps that hit the same
-// cell, or between two of a lane's own eight updates.
+// cell, or between two of a lane's own eight updates.  (Giving each sketch row to one warp and
+// updating with plain load-add-store, which needs no retries and is bit-reproducible, was
+// measured 3.4x slower here: too few warps to hide the shared-memory latency.)
 #include <cuda.h>
 
 #include <algorithm>
@@ -68,7 +70,7 @@ __device__ __forceinline__ float flip(float v, uint32_t signbit)
 __device__ __forceinline__ float lds_f32(uint32_t addr)
 {
     float v;
-    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
 __device__ __forceinline__ float4 lds_f32x4(uint32_t addr)

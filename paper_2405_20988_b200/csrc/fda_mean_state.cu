@@ -18,7 +18,7 @@
 // atomics: warp r owns sketch row r and the 32 lane-private columns of its bins outright,
 // streams the whole vector itself (the other warps' loads of the same bytes hit L1) and
 // updates with plain load-add-store, four indices per lane at a time; equal cells among the
-// four are folded before the stores.  k_sketch_vector (compare-and-swap on bins[cell][C]) is
+// four are folded so that every store to such a cell carries the whole sum.  k_sketch_vector (compare-and-swap on bins[cell][C]) is
 // kept for sketches whose bins do not fit with 32 columns.
 #include <algorithm>
 
@@ -36,7 +36,7 @@ __device__ __forceinline__ float flip(float v, uint32_t signbit)
 __device__ __forceinline__ float lds_f32(uint32_t addr)
 {
     float v;
-    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
 __device__ __forceinline__ uint32_t cas_shared(uint32_t addr, uint32_t expect, uint32_t val)
@@ -252,14 +252,18 @@ __global__ void __launch_bounds__(32 * FDA_MAX_ROWS, 1) k_sketch_vector_rows(con
         const float v0 = flip(a.x, (h.x << 16) & 0x80000000u), v1 = flip(a.y, h.x & 0x80000000u);
         const float v2 = flip(a.z, (h.y << 16) & 0x80000000u), v3 = flip(a.w, h.y & 0x80000000u);
         const float o0 = lds_f32(a0), o1 = lds_f32(a1), o2 = lds_f32(a2), o3 = lds_f32(a3);
-        // stores are issued in order, so a later store to the same cell must carry the earlier values
-        const float w1 = v1 + (a1 == a0 ? v0 : 0.f);
-        const float w2 = v2 + (a2 == a0 ? v0 : 0.f) + (a2 == a1 ? v1 : 0.f);
-        const float w3 = v3 + (a3 == a0 ? v0 : 0.f) + (a3 == a1 ? v1 : 0.f) + (a3 == a2 ? v2 : 0.f);
-        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a0), "f"(o0 + v0) : "memory");
-        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a1), "f"(o1 + w1) : "memory");
-        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a2), "f"(o2 + w2) : "memory");
-        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a3), "f"(o3 + w3) : "memory");
+        // equal cells among the four: every store to such a cell carries the sum of all of them, so
+        // the result does not depend on the order in which the stores land (two stores of one
+        // thread to one shared address were observed to land out of program order on B200)
+        const bool e01 = a0 == a1, e02 = a0 == a2, e03 = a0 == a3, e12 = a1 == a2, e13 = a1 == a3, e23 = a2 == a3;
+        const float t0 = v0 + (e01 ? v1 : 0.f) + (e02 ? v2 : 0.f) + (e03 ? v3 : 0.f);
+        const float t1 = v1 + (e01 ? v0 : 0.f) + (e12 ? v2 : 0.f) + (e13 ? v3 : 0.f);
+        const float t2 = v2 + (e02 ? v0 : 0.f) + (e12 ? v1 : 0.f) + (e23 ? v3 : 0.f);
+        const float t3 = v3 + (e03 ? v0 : 0.f) + (e13 ? v1 : 0.f) + (e23 ? v2 : 0.f);
+        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a0), "f"(o0 + t0) : "memory");
+        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a1), "f"(o1 + t1) : "memory");
+        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a2), "f"(o2 + t2) : "memory");
+        asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(a3), "f"(o3 + t3) : "memory");
     };
 
     // groups of kGroup steps: the loads of the next group are in flight while this one is applied

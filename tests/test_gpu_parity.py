@@ -348,6 +348,49 @@ def test_average_random_and_unaligned(env):
             assert np.array_equal(got[:, d:], w_np[:, d:])
 
 
+def test_average_with_direction_refresh(env):
+    """fda_average_models_xi: the average as before plus xi = (w-bar_new - w_t0_old)/||.||."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(33)
+    with F.FdaContext(0, 0, None, d_max=400_000, K_max=64) as ctx:
+        buf = ctx.new_estimate_buffer()
+        for K, d, off in ((5, 61_706, 0), (8, 300_001, 0), (60, 20_001, 0), (3, 9, 1)):
+            stride = S.row_stride(d) + (1 if off else 0)
+            w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+            w_np = np.zeros((K, stride), dtype=np.float32)
+            w_np[:, :d] = w_t0 + rng.normal(3e-4, 1e-3, size=(K, d)).astype(np.float32)
+            ref_avg = oracle.average(w_np[:, :d])
+            ref_xi = oracle.direction(ref_avg, w_t0)
+            w = torch.from_numpy(w_np).cuda()
+            w0 = torch.from_numpy(w_t0).cuda()
+            xi = torch.full((d + 4,), 9.0, dtype=torch.float32, device="cuda")[off:off + d]
+            ctx.fda_average_models_xi(w[:, :d], w0, xi, None, F.FDA_AVG_BROADCAST | F.FDA_AVG_UNCONDITIONAL)
+            torch.cuda.synchronize()
+            check_average(w0.cpu().numpy(), ref_avg)
+            got = xi.cpu().numpy().astype(np.float64)
+            # the step is a difference of nearby numbers, so xi inherits the fp32 rounding of w-bar
+            # (K sequential adds: at most (K/2 + 2) * 2^-24 |w-bar|) amplified by 1/||step||
+            step_norm = np.linalg.norm(ref_avg - w_t0)
+            tol = (REL * np.maximum(np.abs(ref_xi), 1.0 / np.sqrt(d)) +
+                   (K / 2 + 2) * 2.0 ** -24 * np.maximum(np.abs(ref_avg), np.abs(w_t0)) / step_norm)
+            assert np.all(np.abs(got - ref_xi) <= tol)
+            assert abs(float(np.sum(got * got)) - 1.0) <= 1e-5
+            assert all(np.array_equal(w.cpu().numpy()[k, :d], w0.cpu().numpy()) for k in range(K))
+        # gate closed: nothing is written; zero step: xi becomes 0
+        K, d = 4, 1000
+        w = torch.ones((K, d), dtype=torch.float32, device="cuda")
+        w0 = torch.ones(d, dtype=torch.float32, device="cuda")
+        xi = torch.full((d,), 9.0, dtype=torch.float32, device="cuda")
+        st = torch.zeros((K, 2), dtype=torch.float32, device="cuda")
+        assert ctx.fda_combine_estimate(st, K, 0, 0.0, 1.0, buf).trigger == 0
+        ctx.fda_average_models_xi(w, w0, xi, buf, F.FDA_AVG_BROADCAST)
+        torch.cuda.synchronize()
+        assert bool((xi == 9.0).all())
+        ctx.fda_average_models_xi(w, w0, xi, None, F.FDA_AVG_UNCONDITIONAL)
+        torch.cuda.synchronize()
+        assert not bool(xi.any())
+
+
 # ----------------------------------------------------------------- the five workloads
 def full_round(env, idx, workers_for_oracle=None, check_avg_ranges=None):
     """local state -> combine (both variants, every Theta) -> average; oracle beside it."""

@@ -329,3 +329,18 @@ def test_workload_expectations(idx, mean_sq, ubar_sq):
     assert lin["H"] >= var * (1 - 1e-6)
     assert sk["est"] * (1 + wl.epsilon) == pytest.approx(ub, rel=0.25)
     assert sk["trigger"] and lin["trigger"]
+
+
+def test_direction_heuristic_closed_forms():
+    """xi = (w_new - w_old)/||.|| (Section 3.2): a 3-4-5 step, unit norm, parallelism, zero step."""
+    old = np.array([1.0, 2.0, 3.0, 4.0], dtype=np.float32)
+    new = old.astype(np.float64) + np.array([3.0, 0.0, -4.0, 0.0])
+    assert np.allclose(oracle.direction(new, old), [0.6, 0.0, -0.8, 0.0], rtol=0, atol=1e-15)
+    rng = np.random.default_rng(15)
+    old = rng.normal(size=1000).astype(np.float32)
+    new = old.astype(np.float64) + rng.normal(0, 1e-3, size=1000)
+    xi = oracle.direction(new, old)
+    step = new - old
+    assert np.sum(xi * xi) == pytest.approx(1.0, rel=1e-13)
+    assert xi @ step == pytest.approx(np.linalg.norm(step), rel=1e-13)      # parallel, same sense
+    assert not oracle.direction(old.astype(np.float64), old).any()
