@@ -487,6 +487,37 @@ def test_workload_5_convnextlarge_full_size(env):
                check_avg_ranges=[(0, 50_000), (d // 3, d // 3 + 50_000), (d - 50_001, d)])
 
 
+@pytest.mark.parametrize("l,m", [(3, 100), (8, 1000), (5, 250)])
+def test_vgg16_sized_shape_with_other_sketch_sizes(env, l, m):
+    """A second workload shape: d = 2.6M (the paper's VGG16* row of Table 2), K = 20, smaller and
+    larger sketches than the recommended 5 x 250 (Section 3.3 leaves other sizes open)."""
+    torch, oracle, F = env
+    wl = S.small_workload(seed=11, d=2_600_000, K=20, l=l, m=m, drift="shared", sigma=1e-3,
+                          epsilon=0.06 * (250.0 / m) ** 0.5)
+    w_t0 = S.last_global_model(wl)
+    wbuf = S.worker_models(wl, w_t0, threads=16)
+    xi = S.unit_direction(wl)
+    coeffs = S.hash_coefficients(wl.seed, l)
+    d, K = wl.d, wl.K
+    ks = [0, 9, 19]
+    ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, l, m, workers=ks, threads=3)
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        w, w0, xg, st = gpu_states(torch, F, ctx, wbuf, w_t0, xi)
+        ctx.fda_local_state(w[:, :d], w0, xg, ALL, st)
+        torch.cuda.synchronize()
+        got = st.cpu().numpy()
+        check_states(got, ora, l, m, d, rows=ks)
+        buf = ctx.new_estimate_buffer()
+        for variant in (0, 1):
+            ref = oracle.combine(got, l, m, variant, wl.epsilon, 1e-2)
+            e = ctx.fda_combine_estimate(st, K, variant, np.float32(wl.epsilon), 1e-2, buf).as_dict()
+            tol = check_estimate(e, ref, l)
+            check_trigger(e, ref, 1e-2, tol)
+        ctx.fda_average_models(w[:, :d], w0, buf, F.FDA_AVG_BROADCAST)
+        torch.cuda.synchronize()
+        check_average(w0.cpu().numpy(), oracle.average(wbuf[:, :d]))
+
+
 # ------------------------------------------------------------------ host entry point
 def test_round_host_matches_device_path(env):
     torch, oracle, F = env
