@@ -34,7 +34,8 @@ struct LsParams {
 };
 
 constexpr int kQuadsPerLane = 2;   // float4 loads per lane and tile
-constexpr int kFastThreads = 384;  // block size of the fast sketch kernel
+constexpr int kFastThreads = 640;  // block size of the fast sketch kernel
+constexpr int kFastQuads = 1;      // index quads per lane and tile in the fast sketch kernel (4 updates in flight)
 
 __device__ __forceinline__ float flip(float v, uint32_t signbit)   // signbit: 0 or 0x80000000
 {
@@ -196,8 +197,8 @@ __device__ __forceinline__ void red_shared_add(uint32_t addr, float v)
 
 template <int L, bool LINEAR>
 struct TileRegs {
-    float4 a[kQuadsPerLane], b[kQuadsPerLane], q[kQuadsPerLane];
-    uint2 h[L][kQuadsPerLane];
+    float4 a[kFastQuads], b[kFastQuads], q[kFastQuads];
+    uint2 h[L][kFastQuads];
 };
 
 template <int LWK, int L, bool LINEAR>
@@ -207,7 +208,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) k_local_state_fast(const LsPa
     float *bins = reinterpret_cast<float *>(smem_raw);
 
     constexpr int JS = 32 / LWK;
-    constexpr int TW = JS * kQuadsPerLane * 4;
+    constexpr int TW = JS * kFastQuads * 4;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int kl = lane % LWK, s = lane / LWK;
     const int g = blockIdx.x / p.cpg, c = blockIdx.x % p.cpg;
@@ -233,7 +234,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) k_local_state_fast(const LsPa
 
         auto load_tile = [&](TileRegs<L, LINEAR> &r, int64_t tile) {
 #pragma unroll
-            for (int v = 0; v < kQuadsPerLane; ++v) {
+            for (int v = 0; v < kFastQuads; ++v) {
                 const int64_t jq = tile * TJ + lane_off + (int64_t)v * (JS * 4);
                 if (jq + 3 < p.d) {
                     r.a[v] = __ldg(reinterpret_cast<const float4 *>(wk + jq));
@@ -271,10 +272,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) k_local_state_fast(const LsPa
             const bool more = tile + p.cpg < p.tiles;
             if (more) load_tile(nxt, tile + p.cpg);
 
-            float u[kQuadsPerLane * 4];
+            float u[kFastQuads * 4];
             float pn = 0.f, pp = 0.f;
 #pragma unroll
-            for (int v = 0; v < kQuadsPerLane; ++v) {
+            for (int v = 0; v < kFastQuads; ++v) {
                 u[4 * v + 0] = cur.a[v].x - cur.b[v].x; u[4 * v + 1] = cur.a[v].y - cur.b[v].y;
                 u[4 * v + 2] = cur.a[v].z - cur.b[v].z; u[4 * v + 3] = cur.a[v].w - cur.b[v].w;
                 if (LINEAR) {
@@ -283,18 +284,18 @@ __global__ void __launch_bounds__(kFastThreads, 1) k_local_state_fast(const LsPa
                 }
             }
 #pragma unroll
-            for (int e = 0; e < kQuadsPerLane * 4; ++e) pn = fmaf(u[e], u[e], pn);
+            for (int e = 0; e < kFastQuads * 4; ++e) pn = fmaf(u[e], u[e], pn);
             acc_n += (double)pn;
             if (LINEAR) acc_p += (double)pp;
 
 #pragma unroll
             for (int i = 0; i < L; ++i) {
-                constexpr int NB = kQuadsPerLane * 4;
+                constexpr int NB = kFastQuads * 4;
                 uint32_t addr[NB];
                 float val[NB], old[NB];
                 const uint32_t rowaddr = col_addr + (uint32_t)i * row_bytes;
 #pragma unroll
-                for (int v = 0; v < kQuadsPerLane; ++v) {
+                for (int v = 0; v < kFastQuads; ++v) {
                     const uint32_t hx = cur.h[i][v].x, hy = cur.h[i][v].y;
                     addr[4 * v + 0] = rowaddr + ((hx & 0x7fffu) << bshift);
                     addr[4 * v + 1] = rowaddr + (((hx >> 16) & 0x7fffu) << bshift);
@@ -494,7 +495,7 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
     const int threads = fast ? kFastThreads : (sketch ? 1024 : 512);
     const int blocks_per_sm = sketch ? 1 : 2;
     const int js = 32 / lwk;
-    const int64_t tile_j = (int64_t)(threads / 32) * js * kQuadsPerLane * 4;
+    const int64_t tile_j = (int64_t)(threads / 32) * js * (fast ? kFastQuads : kQuadsPerLane) * 4;
     p.tiles = (d + tile_j - 1) / tile_j;
     int64_t cpg = (int64_t)ctx->n_sm * blocks_per_sm / groups;
     if (cpg < 1) cpg = 1;

@@ -115,21 +115,28 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
     }
 }
 
-// states[k][0..1] = sum over blocks (block order, fp64); every sketch slot is written as 0.
+// states[k][0..1] = sum over blocks in fp64 (one warp per value: lanes take blocks b = lane,
+// lane + 32, ..., then a fixed shuffle tree, so the result is reproducible); every sketch slot
+// is written as 0.
 __global__ void k_finalize_linear(const double *__restrict__ part_np, int K, int blocks, int slen,
                                   uint32_t flags, bool have_xi, float *__restrict__ states)
 {
-    const int64_t total = (int64_t)K * slen;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-         t += (int64_t)gridDim.x * blockDim.x) {
-        const int k = (int)(t / slen), e = (int)(t % slen);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t v = warp; v < (int64_t)K * 2; v += nwarps) {
+        const int k = (int)(v / 2), e = (int)(v % 2);
+        const bool on = e == 0 ? (flags & FDA_STATE_NORM) != 0 : ((flags & FDA_STATE_LINEAR) != 0 && have_xi);
         double acc = 0.0;
-        const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0
-                      : (e == 1) ? ((flags & FDA_STATE_LINEAR) != 0 && have_xi) : false;
         if (on)
-            for (int b = 0; b < blocks; ++b) acc += part_np[((size_t)b * K + k) * 2 + e];
-        states[t] = (float)acc;
+            for (int b = lane; b < blocks; b += 32) acc += part_np[((size_t)b * K + k) * 2 + e];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) states[(size_t)k * slen + e] = (float)acc;
     }
+    const int64_t cells = (int64_t)K * (slen - 2);
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < cells; t += (int64_t)gridDim.x * blockDim.x)
+        states[(t / (slen - 2)) * slen + 2 + t % (slen - 2)] = 0.f;
 }
 
 template <int KPW>

@@ -11,7 +11,7 @@
 // bulk copies (cp.async.bulk) were measured at one copy per 230-420 clocks per SM, which
 // starves tiles made of 30+ short rows; 16-byte cp.async from all threads loads the same
 // pipe the scatter needs.  Hence tiled tensor copies: one cp.async.bulk.tensor.2d brings a
-// [workers x BX] box, with BX = 4 (mod 32) floats so that the dense box rows fall on
+// [workers x BX] box, with BX/4 odd so that the dense box rows fall on
 // different banks, and zero-fills everything outside the tensor (ragged end, missing rows).
 // No multicast is used anywhere.
 //
@@ -25,10 +25,10 @@
 // consumer warp has released the stage.  Every wait is bounded: when it runs out the thread
 // raises the context's error word and stops waiting, so the kernel always returns.
 //
-// Updates.  Eight shared-memory updates per lane are in flight (eight loads, eight adds,
-// eight compare-and-swaps); an update whose compare-and-swap lost a race is redone with an
+// Updates.  Four shared-memory updates per lane are in flight (four loads, four adds, four
+// compare-and-swaps); an update whose compare-and-swap lost a race is redone with an
 // atomic add.  Lanes own their column, so races only occur between warps that hit the same
-// cell, or between two of a lane's own eight updates.  (Giving each sketch row to one warp and
+// cell, or between two of a lane's own four updates.  (Giving each sketch row to one warp and
 // updating with plain load-add-store, which needs no retries and is bit-reproducible, was
 // measured 3.4x slower here: too few warps to hide the shared-memory latency.)
 #include <cuda.h>
@@ -39,7 +39,6 @@
 
 namespace {
 
-constexpr int kMaxStages = 3;
 constexpr int kMaxThreads = 1024;
 constexpr int kMaxUnits = 64;
 constexpr int kMaxBoxes = 4;                   // tensor boxes per tile
@@ -52,7 +51,7 @@ struct StagedParams {
     int l, m;
     int Kg, groups;
     int roles, rows_per_role;        // role r owns rows [r*rows_per_role, min(l, ...))
-    int bx, nb;                      // box width (floats, = 4 mod 32) and boxes per tile
+    int bx, nb;                      // box width (floats, bx/4 odd) and boxes per tile
     int stages;                      // depth of the shared-memory ring
     int64_t tiles;                   // ceil(d / (bx*nb))
     uint32_t wbox_bytes, vbox_bytes, hbox_bytes;   // 128-byte aligned sizes of one box
@@ -120,6 +119,38 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(mbar) : "memory");
 }
 
+// N updates of lane-private cells: N loads, N adds, N compare-and-swaps in flight; the ones that
+// lost a race are redone with an atomic add, one per lane and round, so that the lanes of a
+// warp share the retry instruction whichever of their updates failed.
+template <int N>
+__device__ __forceinline__ void apply_updates(const uint32_t (&addr)[N], const float (&val)[N])
+{
+    float old[N];
+    uint32_t got[N];
+#pragma unroll
+    for (int e = 0; e < N; ++e) old[e] = lds_f32(addr[e]);
+    uint32_t diff = 0;
+#pragma unroll
+    for (int e = 0; e < N; ++e) {
+        got[e] = cas_shared(addr[e], __float_as_uint(old[e]), __float_as_uint(old[e] + val[e]));
+        diff |= got[e] ^ __float_as_uint(old[e]);
+    }
+    if (diff) {
+        uint32_t lost = 0;
+#pragma unroll
+        for (int e = 0; e < N; ++e) lost |= (got[e] != __float_as_uint(old[e])) ? (1u << e) : 0u;
+        while (lost) {
+            uint32_t a = addr[0];
+            float v = val[0];
+#pragma unroll
+            for (int e = 1; e < N; ++e)
+                if ((lost & ((1u << e) - 1u)) == 0 && (lost & (1u << e))) { a = addr[e]; v = val[e]; }
+            red_shared_add(a, v);
+            lost &= lost - 1u;
+        }
+    }
+}
+
 // Shared-memory plan (bytes from the start of dynamic shared memory):
 //   [0, 64)                  mbarriers: full[s] at 8*s, empty[s] at 32 + 8*s
 //   [128, 128 + bins_bytes)  bins[local cell][32]
@@ -128,6 +159,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 //        W0 [bx] floats            at nb*wbox_bytes + b*vbox_bytes
 //        XI [bx] floats            at nb*(wbox_bytes + vbox_bytes) + b*vbox_bytes
 //        H  [rows_per_role][bx] uint32    at nb*(wbox_bytes + 2*vbox_bytes) + b*hbox_bytes
+// A lane takes one index quad per pass: four updates in flight per lane and sketch row.  Two
+// quads (eight in flight) or two rows at once (sixteen) were measured slower: what pays is
+// many warps with short windows between load and compare-and-swap, which keeps the share of
+// lost races down.
 template <int LWK, bool LINEAR>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap tm_w,
@@ -136,7 +171,8 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int JS = 32 / LWK;
-    constexpr int NB = 8;                       // updates in flight per lane
+    constexpr int QPL = 1;                      // index quads per lane and pass
+    constexpr int NB = 4 * QPL;                 // updates in flight per lane
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const int ncons = nwarps - 1;               // consumer warps
     const int cw = warp - 1;                    // consumer index (-1: producer)
@@ -186,7 +222,7 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
     const uint32_t col_addr = bins_addr + (uint32_t)lane * 4u;
     const int qpb = bx / 4;                                        // quads per box
     const int quads = qpb * nb;                                    // quads per tile
-    const int quads_per_pass = ncons * JS * 2;
+    const int quads_per_pass = ncons * JS * QPL;
     const int passes = (quads + quads_per_pass - 1) / quads_per_pass;
 
     // one staged tile -> bins (+ norm / projection partials); consumer warps only
@@ -194,12 +230,12 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
         if (!active) return;
         for (int ps = 0; ps < passes; ++ps) {
             float u[NB];
-            uint32_t haddr[2];
+            uint32_t haddr[QPL];
             bool any = false;
             float pp = 0.f;
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-                const int q = (ps * ncons + cw) * (JS * 2) + v * JS + s;         // quad inside the tile
+            for (int v = 0; v < QPL; ++v) {
+                const int q = (ps * ncons + cw) * (JS * QPL) + v * JS + s;       // quad inside the tile
                 const bool in = q < quads;
                 any |= in;
                 const int b = in ? q / qpb : 0, xq = in ? q - b * qpb : 0;
@@ -225,11 +261,9 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                 acc_n += (double)pn;
                 if (LINEAR) acc_p += (double)pp;
             }
-            for (int i = 0; i < rows; ++i) {
-                uint32_t addr[NB], got[NB];
-                float val[NB], old[NB];
+            auto row_updates = [&](int i, uint32_t *addr, float *val) {
 #pragma unroll
-                for (int v = 0; v < 2; ++v) {
+                for (int v = 0; v < QPL; ++v) {
                     // 4 table words of this quad: cell byte offset | sign << 31 (u = 0 where the quad is absent)
                     uint32_t h[4];
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -240,30 +274,13 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                         val[4 * v + e] = flip(u[4 * v + e], h[e] & 0x80000000u);
                     }
                 }
-#pragma unroll
-                for (int e = 0; e < NB; ++e) old[e] = lds_f32(addr[e]);
-                uint32_t diff = 0;          // non-zero when some compare-and-swap of the eight lost a race
-#pragma unroll
-                for (int e = 0; e < NB; ++e) {
-                    got[e] = cas_shared(addr[e], __float_as_uint(old[e]), __float_as_uint(old[e] + val[e]));
-                    diff |= got[e] ^ __float_as_uint(old[e]);
-                }
-                if (diff) {
-                    // redo the lost ones, one per lane and round, so that the lanes of a warp share
-                    // the retry instruction whichever of their eight updates failed
-                    uint32_t lost = 0;
-#pragma unroll
-                    for (int e = 0; e < NB; ++e) lost |= (got[e] != __float_as_uint(old[e])) ? (1u << e) : 0u;
-                    while (lost) {
-                        uint32_t a = addr[0];
-                        float v = val[0];
-#pragma unroll
-                        for (int e = 1; e < NB; ++e)
-                            if ((lost & ((1u << e) - 1u)) == 0 && (lost & (1u << e))) { a = addr[e]; v = val[e]; }
-                        red_shared_add(a, v);
-                        lost &= lost - 1u;
-                    }
-                }
+            };
+            int i = 0;
+            for (; i < rows; ++i) {
+                uint32_t addr[NB];
+                float val[NB];
+                row_updates(i, addr, val);
+                apply_updates<NB>(addr, val);
             }
         }
     };
@@ -473,13 +490,26 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
         return (size_t)nb * (align128((size_t)p.Kg * bx * 4) + 2 * align128((size_t)bx * 4) +
                              align128((size_t)rows * bx * 4));
     };
+    // Among the (box width, boxes per tile) pairs that fit: first as many consumer warps as the
+    // tile can keep busy (counted up to 28: beyond that a larger tile pays more), then the
+    // largest tile.  One quad per lane and pass; box width / 4 odd keeps the box rows on
+    // different banks.
+    const int js_sel = 32 / lwk;
+    auto warps_for = [&](int tile_indices) -> int {
+        const int q = tile_indices / 4, cap = kMaxThreads / 32 - 1;
+        const int passes = (q + cap * js_sel - 1) / (cap * js_sel);
+        return (q + passes * js_sel - 1) / (passes * js_sel);
+    };
     auto best_tile = [&](int rows, int stages, int *bx_out, int *nb_out) -> int {
-        int best = 0;
+        int best = 0, best_w = 0;
         if (budget <= (size_t)rows * row_bins) return 0;
         const size_t room = (budget - (size_t)rows * row_bins) / stages;
-        for (int bx = 228; bx >= 36; bx -= 32)
-            for (int nb = kMaxBoxes; nb >= 1; --nb)
-                if (stage_size(rows, bx, nb) <= room && bx * nb > best) { best = bx * nb; *bx_out = bx; *nb_out = nb; }
+        for (int bx = 252; bx >= 36; bx -= 8)
+            for (int nb = kMaxBoxes; nb >= 1; --nb) {
+                if (stage_size(rows, bx, nb) > room) continue;
+                const int t = bx * nb, wv = std::min(warps_for(t), 28);
+                if (wv > best_w || (wv == best_w && t > best)) { best = t; best_w = wv; *bx_out = bx; *nb_out = nb; }
+            }
         return best;
     };
     int rows_cap = 0, bx = 0, nb = 0;
@@ -492,11 +522,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     if (rows_cap < ctx->l) return cudaErrorNotSupported;
     p.roles = 1;
     p.rows_per_role = ctx->l;
-    p.stages = 2;
-    for (int st = kMaxStages; st > 2; --st) {
-        int bx3 = 0, nb3 = 0;
-        if (best_tile(p.rows_per_role, st, &bx3, &nb3) >= 512) { p.stages = st; break; }
-    }
+    p.stages = 2;      // deeper rings were measured slower (smaller tiles, same latency cover)
     const int tile = best_tile(p.rows_per_role, p.stages, &bx, &nb);
     p.bx = bx; p.nb = nb;
     p.tiles = (d + tile - 1) / tile;
@@ -506,15 +532,8 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     const int units = p.roles * p.groups;
     if (units > kMaxUnits || units > ctx->n_sm) return cudaErrorNotSupported;
 
-    // consumer warps: the fewest passes over the tile's quads with at most 31 warps, then the
-    // fewest warps that still need no more passes (throughput follows the number of busy warps)
-    const int js = 32 / lwk, quads = tile / 4;
-    int ncons = kMaxThreads / 32 - 1;
-    {
-        int passes = (quads + ncons * js * 2 - 1) / (ncons * js * 2);
-        ncons = (quads + passes * js * 2 - 1) / (passes * js * 2);
-        if (ncons < 4) ncons = 4;
-    }
+    int ncons = warps_for(tile);
+    if (ncons < 4) ncons = 4;
     const int threads = (ncons + 1) * 32;
 
     // blocks per unit in proportion to the rows the unit scatters

@@ -296,24 +296,30 @@ __global__ void __launch_bounds__(32 * FDA_MAX_ROWS, 1) k_sketch_vector_rows(con
     }
 }
 
-// mean_state[e] = (sum over blocks, block order, fp64) [/ K for the two scalars]
+// mean_state[e] = sum over blocks in fp64 [/ K for the two scalars].  Warp 0 and 1 of block 0
+// reduce the scalar partials (lanes stride the blocks, fixed shuffle tree); the cells are summed
+// in block order by one thread each.
 __global__ void k_finalize_mean(const float *__restrict__ part_sk, const double *__restrict__ part_np,
                                 int np_blocks, int sk_blocks, int lm, int K, uint32_t flags, bool have_xi,
                                 float *__restrict__ mean_state)
 {
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= 2 + lm) return;
-    double acc = 0.0;
-    if (e < 2) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && warp < 2) {
+        const int e = warp;
         const bool on = e == 0 ? (flags & FDA_STATE_NORM) != 0 : ((flags & FDA_STATE_LINEAR) != 0 && have_xi);
-        if (on) {
-            for (int b = 0; b < np_blocks; ++b) acc += part_np[(size_t)b * 2 + e];
-            acc /= (double)K;
-        }
-    } else if (flags & FDA_STATE_SKETCH) {
-        for (int b = 0; b < sk_blocks; ++b) acc += (double)part_sk[(size_t)b * lm + (e - 2)];
+        double acc = 0.0;
+        if (on)
+            for (int b = lane; b < np_blocks; b += 32) acc += part_np[(size_t)b * 2 + e];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) mean_state[e] = (float)(acc / (double)K);
     }
-    mean_state[e] = (float)acc;
+    const int cell = blockIdx.x * blockDim.x + threadIdx.x;
+    if (cell >= lm) return;
+    double acc = 0.0;
+    if (flags & FDA_STATE_SKETCH)
+        for (int b = 0; b < sk_blocks; ++b) acc += (double)part_sk[(size_t)b * lm + cell];
+    mean_state[2 + cell] = (float)acc;
 }
 
 int ilog2(int v) { int r = 0; while ((1 << (r + 1)) <= v) ++r; return r; }
@@ -392,7 +398,7 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
         }
         if (e != cudaSuccess) return e;
     }
-    const int n = 2 + ctx->lm;
+    const int n = ctx->lm > 64 ? ctx->lm : 64;        // at least two warps for the scalars
     k_finalize_mean<<<(n + 255) / 256, 256, 0, s>>>(ctx->part_sk, ctx->part_np, (int)nblk, sk_blocks, ctx->lm, K,
                                                    flags, linear, mean_state);
     return cudaGetLastError();
