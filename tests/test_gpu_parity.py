@@ -518,6 +518,47 @@ def test_vgg16_sized_shape_with_other_sketch_sizes(env, l, m):
         check_average(w0.cpu().numpy(), oracle.average(wbuf[:, :d]))
 
 
+def test_largest_supported_dimension(env):
+    """d just below 2^31 (the limit of fda_create), ragged, one worker, one sketch row: 64-bit
+    offsets, the top of the hash key range and the last partial tile.  The drift is non-zero only
+    in three windows (start, middle, end) so that every cell can be traced to a few indices."""
+    torch, oracle, F = env
+    d, l, m = (1 << 31) - 4097, 1, 250
+    rng = np.random.default_rng(99)
+    coeffs = rand_coeffs(rng, l)
+    w = torch.zeros((1, d), dtype=torch.float32, device="cuda")
+    w0 = torch.zeros(d, dtype=torch.float32, device="cuda")
+    windows = [(0, 70_001), (d // 2 - 33_333, d // 2 + 33_334), (d - 100_003, d)]
+    host = []
+    for lo, hi in windows:
+        v = rng.normal(0, 1e-3, size=hi - lo).astype(np.float32)
+        base = rng.normal(0, 0.05, size=hi - lo).astype(np.float32)
+        w[0, lo:hi] = torch.from_numpy(base + v).cuda()
+        w0[lo:hi] = torch.from_numpy(base).cuda()
+        host.append((lo, hi, (base + v).astype(np.float32), base))
+    # oracle on the windows only (the rest contributes exactly zero): same sums, hash keys offset
+    norm, sk = 0.0, np.zeros(m)
+    for lo, hi, wv, bv in host:
+        u = wv.astype(np.float64) - bv.astype(np.float64)
+        norm += float(np.sum(u * u))
+        b, sg = oracle.hash_dump(coeffs, l, m, lo, hi - lo)
+        np.add.at(sk, b[0], sg[0] * u)
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=1) as ctx:
+        st = torch.empty((1, ctx.state_len), dtype=torch.float32, device="cuda")
+        ctx.fda_local_state(w, w0, None, 1 | 4, st)
+        mean = torch.empty(ctx.state_len, dtype=torch.float32, device="cuda")
+        ctx.fda_mean_state(w, w0, None, 1 | 4, mean)
+        torch.cuda.synchronize()
+        ref = np.concatenate([[norm, 0.0], sk])[None]
+        check_states(st.cpu().numpy(), ref, l, m, d)
+        check_states(mean.cpu().numpy()[None], ref, l, m, d)
+        ctx.fda_average_models(w, w0, None, F.FDA_AVG_UNCONDITIONAL)       # K = 1: w_t0 becomes w bit for bit
+        torch.cuda.synchronize()
+        for lo, hi, wv, _ in host:
+            assert np.array_equal(w0[lo:hi].cpu().numpy(), wv)
+        assert float(w0[70_001:d // 2 - 33_333].abs().max()) == 0.0
+
+
 # ------------------------------------------------------------------ host entry point
 def test_round_host_matches_device_path(env):
     torch, oracle, F = env
