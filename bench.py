@@ -37,10 +37,11 @@ UNIT = "params*workers/s"
 SKETCH_STATE = 1 | 4      # SketchFDA local state (Theorem 1): squared norm + AMS sketch
 LINEAR_STATE = 1 | 2      # LinearFDA local state (Theorem 2): squared norm + projection
 FALLBACK_HBM_GBS = 6650.0
+SMEM_CAS_UPDATES_PER_CLK_SM = 6.8     # measured on B200: bare fp32 shared-memory atomicAdd loop, 1024 threads
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
 # capture summarised under profiles/ (None: not captured for the kernel as it stands).
-LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: None, 5: 11_076_100_000}
+LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: 5_164_300_000, 5: 11_076_300_000}
 
 
 def measured_hbm_peak():
@@ -287,6 +288,7 @@ def run_ours(args, rank, world, local_rank):
     out = None
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
+        n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
         algo_bytes = 4.0 * (K * d + d + K * slen)            # w, w_t0 read; states written
         lin_bytes = 4.0 * (K * d + 2 * d + K * slen)         # + xi
         achieved = algo_bytes / (ls_ms * 1e-3) / 1e9
@@ -324,6 +326,14 @@ def run_ours(args, rank, world, local_rank):
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "algorithmic_bytes": algo_bytes,
                          "traffic": LOCAL_STATE_TRAFFIC_BYTES.get(args.workload)},
+            # what really binds the sketch pass: fp32 updates of shared-memory bins, which are
+            # compare-and-swap loops on this hardware (measured ceiling 6.8 updates/clk/SM)
+            "secondary_roofline": {"bound": "smem_cas", "unit": "updates/s",
+                                   "achieved": K * d * wl.l / (ls_ms * 1e-3),
+                                   "peak": SMEM_CAS_UPDATES_PER_CLK_SM * n_sm * (clocks.get("sm_mhz") or 1965.0) * 1e6,
+                                   "frac": K * d * wl.l / (ls_ms * 1e-3) /
+                                           (SMEM_CAS_UPDATES_PER_CLK_SM * n_sm * (clocks.get("sm_mhz") or 1965.0) * 1e6),
+                                   "note": "peak = microbenchmarked fp32 atomicAdd rate on lane-private columns"},
             "cpu_baseline": cpu,
             "e2e": None if not e2e_times else
                    {"value": job_value(world, K * d, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d,
