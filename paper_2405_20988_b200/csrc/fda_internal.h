@@ -31,6 +31,14 @@ struct fda_ctx {
     size_t part_np_doubles = 0;
     int max_blocks = 0;
     float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
+    // tensor maps of the last staged launch (encoding four maps costs several microseconds of
+    // host time, which matters for small models); valid while the key below matches
+    alignas(64) unsigned char tmap_cache[4][128] = {};
+    struct {
+        const void *w = nullptr, *w_t0 = nullptr, *xi = nullptr;
+        int64_t row_stride = 0, d = 0;
+        int K = 0, bx = 0, Kg = 0;
+    } tmap_key;
     unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
     // staging for fda_round_host (lazy)
     float *stage_w = nullptr, *stage_w_t0 = nullptr, *stage_xi = nullptr, *stage_states = nullptr;

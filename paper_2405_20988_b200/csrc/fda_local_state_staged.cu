@@ -555,17 +555,26 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     if ((size_t)blocks * p.part_pitch > ctx->part_sk_floats || blocks > ctx->max_blocks)
         return cudaErrorNotSupported;
 
-    // tensor maps: w [K][d], w_t0 / xi [1][d], hash table [l][tab_stride]
-    CUtensorMap maps[4];
-    const uint64_t vec_pitch = (uint64_t)align128((size_t)d * 4);
-    bool ok = make_map(&maps[0], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w, (uint64_t)d, (uint64_t)K,
-                       (uint64_t)row_stride * 4, (uint32_t)bx, (uint32_t)p.Kg);
-    ok = ok && make_map(&maps[1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w_t0, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
-    ok = ok && make_map(&maps[2], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, xi_used ? xi_used : w_t0, (uint64_t)d, 1,
-                        vec_pitch, (uint32_t)bx, 1);
-    ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT32, ctx->tab32, (uint64_t)ctx->tab_stride,
-                        (uint64_t)ctx->l, (uint64_t)ctx->tab_stride * 4, (uint32_t)bx, (uint32_t)p.rows_per_role);
-    if (!ok) return cudaErrorNotSupported;
+    // tensor maps: w [K][d], w_t0 / xi [1][d], hash table [l][tab_stride]; reused from the last
+    // call when pointers and shapes are the same
+    static_assert(sizeof(CUtensorMap) <= 128, "tensor map does not fit its cache slot");
+    CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(ctx->tmap_cache);
+    auto &key = ctx->tmap_key;
+    const void *xi_key = xi_used ? (const void *)xi_used : (const void *)w_t0;
+    if (!(key.w == w && key.w_t0 == w_t0 && key.xi == xi_key && key.row_stride == row_stride && key.d == d &&
+          key.K == K && key.bx == bx && key.Kg == p.Kg)) {
+        key.w = nullptr;
+        const uint64_t vec_pitch = (uint64_t)align128((size_t)d * 4);
+        bool ok = make_map(&maps[0], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w, (uint64_t)d, (uint64_t)K,
+                           (uint64_t)row_stride * 4, (uint32_t)bx, (uint32_t)p.Kg);
+        ok = ok && make_map(&maps[1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w_t0, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
+        ok = ok && make_map(&maps[2], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, xi_key, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
+        ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT32, ctx->tab32, (uint64_t)ctx->tab_stride,
+                            (uint64_t)ctx->l, (uint64_t)ctx->tab_stride * 4, (uint32_t)bx, (uint32_t)p.rows_per_role);
+        if (!ok) return cudaErrorNotSupported;
+        key.w = w; key.w_t0 = w_t0; key.xi = xi_key; key.row_stride = row_stride; key.d = d;
+        key.K = K; key.bx = bx; key.Kg = p.Kg;
+    }
 
     size_t smem = 128 + (size_t)p.rows_per_role * row_bins + (size_t)p.stages * stage_size(p.rows_per_role, bx, nb);
     const size_t smem_min = 128 + (size_t)(ncons + 1) * lwk * 2 * sizeof(double);     // reduction scratch
