@@ -30,7 +30,7 @@ k_average(float *w, int64_t row_stride, int K, int64_t d, float *__restrict__ w_
 #pragma unroll
                 for (int b = 0; b < kBatch; ++b)
                     if (k0 + b < K)
-                        v[b] = *reinterpret_cast<const float4 *>(w + (size_t)(k0 + b) * row_stride + q * 4);
+                        v[b] = __ldcs(reinterpret_cast<const float4 *>(w + (size_t)(k0 + b) * row_stride + q * 4));
 #pragma unroll
                 for (int b = 0; b < kBatch; ++b)
                     if (k0 + b < K) { acc.x += v[b].x; acc.y += v[b].y; acc.z += v[b].z; acc.w += v[b].w; }
@@ -42,10 +42,10 @@ k_average(float *w, int64_t row_stride, int K, int64_t d, float *__restrict__ w_
                 *reinterpret_cast<float4 *>(xi_out + q * 4) = dl;
                 dsq += (double)(dl.x * dl.x + dl.y * dl.y + dl.z * dl.z + dl.w * dl.w);
             }
-            *reinterpret_cast<float4 *>(w_t0 + q * 4) = acc;
+            __stcs(reinterpret_cast<float4 *>(w_t0 + q * 4), acc);
             if (broadcast)
                 for (int k = 0; k < K; ++k)
-                    *reinterpret_cast<float4 *>(w + (size_t)k * row_stride + q * 4) = acc;
+                    __stcs(reinterpret_cast<float4 *>(w + (size_t)k * row_stride + q * 4), acc);
         }
     }
     // scalar path: everything when !VEC, the d % 4 tail otherwise
