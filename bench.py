@@ -37,6 +37,8 @@ UNIT = "params*workers/s"
 SKETCH_STATE = 1 | 4      # SketchFDA local state (Theorem 1): squared norm + AMS sketch
 LINEAR_STATE = 1 | 2      # LinearFDA local state (Theorem 2): squared norm + projection
 FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 << 20
+NOMINAL_HBM_GBS = 8000.0               # the data-sheet figure, quoted beside the measured copy rate
 SMEM_CAS_UPDATES_PER_CLK_SM = 6.8     # measured on B200: bare fp32 shared-memory atomicAdd loop, 1024 threads
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
@@ -196,6 +198,9 @@ def run_ours(args, rank, world, local_rank):
         # the sync of the previous step made all models equal: put the drifted models back
         w.copy_(w_src)
         w0.copy_(w0_src)
+        return step_events()
+
+    def step_events():
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         ev[0].record(stream)
         ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
@@ -259,7 +264,39 @@ def run_ours(args, rank, world, local_rank):
             mean_ms.append(e0.elapsed_time(e1))
     mean_ms = float(np.mean(mean_ms))
     mean_est = ctx.fda_combine_estimate(mean_state.view(1, -1), 1, F.FDA_VARIANT_SKETCH, eps, theta, est_buf).as_dict()
+    # ---- a kernel that only reads, on the same tensor (yardstick for the streaming kernels) ----
+    probe_out = torch.zeros(1, dtype=torch.float32, device=dev)
+    probe_ms = []
+    for it in range(3 + 10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.fda_debug_read_probe(w, probe_out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if it >= 3:
+            probe_ms.append(e0.elapsed_time(e1))
+    probe_gbs = 4.0 * w.numel() / (float(np.mean(probe_ms)) * 1e-3) / 1e9
+
+    # ---- cold-L2 timing for models that fit in L2 (the restoring copy leaves them cached) ----
+    cold = None
+    if 4 * K * stride < 2 * L2_BYTES:
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+        cold_parts = []
+        for it in range(3 + 10):
+            w.copy_(w_src)
+            w0.copy_(w0_src)
+            flush.zero_()
+            ev = step_events()
+            torch.cuda.synchronize()
+            if it >= 3:
+                cold_parts.append([ev[i].elapsed_time(ev[i + 1]) for i in range(3)])
+        cp = np.array(cold_parts).mean(axis=0)
+        cold = {"local_state": float(cp[0]), "combine": float(cp[1]), "average": float(cp[2]),
+                "note": "a %d MB buffer written between the restoring copy and the step" % (2 * L2_BYTES >> 20)}
+        del flush
+
     step_ms = float(parts.sum(axis=1).mean())
+    step_all = parts.sum(axis=1)
     if dist:
         step_ms = max_over_ranks(step_ms, dist, dev)
     ls_ms, cb_ms, av_ms = (float(x) for x in parts.mean(axis=0))
@@ -297,11 +334,16 @@ def run_ours(args, rank, world, local_rank):
             d_s = cpu_sample_size(wl, cores)
             threads = min(cores, K)
             dt, _ = oracle_step_on_sample(wl, w_pin.numpy(), w_t0_np, xi_np, coeffs, d_s, threads)
+            d_1 = max(4096, d_s // max(1, threads))
+            dt1, _ = oracle_step_on_sample(wl, w_pin.numpy(), w_t0_np, xi_np, coeffs, d_1, 1)
             cpu = {"value": K * d_s / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-                   "sample": "all %d workers x first %d of %d indices, one whole step, %.1f s" % (K, d_s, d, dt)}
+                   "sample": "all %d workers x first %d of %d indices, one whole step, %.1f s" % (K, d_s, d, dt),
+                   "single_thread": {"value": K * d_1 / dt1, "cores": 1,
+                                     "sample": "first %d indices, %.1f s" % (d_1, dt1)}}
         out = {
             "metric": METRIC, "value": job_value(world, K * d, step_ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
+            "ms_per_step_median": float(np.median(step_all)), "ms_per_step_best": float(step_all.min()),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": "%d:%s d=%d K=%d sketch=%dx%d eps=%.4f theta=%g" %
@@ -311,9 +353,13 @@ def run_ours(args, rank, world, local_rank):
                              "each step, outside the timed events" % (4 * K * d / 1e9),
                        "multi_gpu": "replicas only"},
             "kernels_ms": {"local_state": ls_ms, "combine": cb_ms, "average": av_ms},
+            "kernels_ms_cold_l2": cold,
+            "read_probe": {"gbs": probe_gbs, "frac_of_peak": probe_gbs / peak,
+                           "note": "fda_debug_read_probe over the model tensor: a kernel that only reads"},
             "local_state_only": {"value": K * d / (ls_ms * 1e-3), "unit": UNIT},
             "average_only": {"gbs": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9,
-                             "frac_of_peak": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9 / peak},
+                             "frac_of_peak": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9 / peak,
+                             "frac_of_nominal_8tbs": 4.0 * (2 * K * d + d) / (av_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
             "linear_local_state": {"ms": lin_ms, "value": K * d / (lin_ms * 1e-3), "unit": UNIT,
                                    "gbs": lin_bytes / (lin_ms * 1e-3) / 1e9,
                                    "frac_of_peak": lin_bytes / (lin_ms * 1e-3) / 1e9 / peak, "H": lin_est["H"]},
@@ -325,6 +371,7 @@ def run_ours(args, rank, world, local_rank):
             "roofline": {"kernel": "k_local_state_fast" if args.workload == 4 else "k_local_state_staged", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "algorithmic_bytes": algo_bytes,
+                         "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
                          "traffic": LOCAL_STATE_TRAFFIC_BYTES.get(args.workload)},
             # what really binds the sketch pass: fp32 updates of shared-memory bins, which are
             # compare-and-swap loops on this hardware (measured ceiling 6.8 updates/clk/SM)

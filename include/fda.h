@@ -202,6 +202,18 @@ fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets
                           int8_t *signs, void *stream);
 
 /*
+ * Read-only bandwidth probe (the paper has no counterpart): streams src[0..n) once with the
+ * access pattern of the bandwidth-bound kernels and writes the sum of its elements to
+ * *sum_out (device, one float; fp32 per thread, fp64 across threads, fixed order).  Timing
+ * this call gives the rate a kernel that only reads reaches on the device, which is the
+ * yardstick quoted beside the local-state and averaging kernels.  src need not be aligned.
+ * Uses the context's partial-sum scratch: not concurrent with other calls on the context.
+ * Errors: INVALID_ARG (NULL, n < 1), CUDA.
+ */
+fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float *sum_out,
+                                void *stream);
+
+/*
  * Local state without a context and without any allocation.  (The paper has no counterpart
  * to this call; it exists for the way some programs have to use the library.)
  *

@@ -332,4 +332,16 @@ fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets
     return FDA_OK;
 }
 
+fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float *sum_out, void *stream)
+{
+    if (!ctx) return FDA_ERR_INVALID_ARG;
+    if (!src || !sum_out || n < 1)
+        return fail(ctx, FDA_ERR_INVALID_ARG, "fda_debug_read_probe: argument out of range");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, FDA_ERR_CUDA, "fda_debug_read_probe: cannot select device");
+    cudaError_t e = fda_launch_read_probe(ctx, src, n, sum_out, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_debug_read_probe");
+    return FDA_OK;
+}
+
 }  // extern "C"

@@ -50,6 +50,8 @@ struct fda_ctx {
 
 // ---- launchers (each returns the cudaError_t of its launches) -------------------------
 cudaError_t fda_launch_build_table(const fda_ctx *ctx, cudaStream_t s);
+cudaError_t fda_launch_read_probe(const fda_ctx *ctx, const float *src, int64_t n, float *sum_out,
+                                  cudaStream_t s);
 cudaError_t fda_launch_debug_hash(const fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets,
                                   int8_t *signs, cudaStream_t s);
 cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K,

@@ -1,7 +1,8 @@
 // Local-state pass without the sketch: ||u^(k)||^2 and <xi,u^(k)> only (Section 3, local
 // state; Section 3.2, LinearFDA).  Pure streaming: K*d + 2*d floats are read once.
 //
-// A block walks index tiles; w_t0 and xi of a tile are parked in shared memory once and every
+// A block walks index tiles; w_t0 and xi of a tile are parked in shared memory once (the next
+// tile's copy runs asynchronously under the current tile's row streaming) and every
 // warp then streams the rows of "its" workers (k = warp, warp + NW, ...) with coalesced
 // 128-bit loads, several in flight per lane.  With fewer workers than warps, several warps
 // share a worker and split the tile's chunks between them.  fp32 partial sums cover one tile (at most 64
@@ -11,10 +12,20 @@
 
 namespace {
 
-constexpr int kTile = 2048;           // indices per tile
+constexpr int kTile = 4096;           // indices per tile
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kChunks = kTile / 128;  // 128 indices = one float4 per lane
+
+__device__ __forceinline__ void cp_async16(float *dst_shared, const float *src)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(dst_shared);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(a), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
 
 template <int KPW, bool LINEAR, bool VEC>
 __global__ void __launch_bounds__(kThreads)
@@ -22,8 +33,10 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
                      const float *__restrict__ w_t0, const float *__restrict__ xi, int64_t tiles,
                      double *__restrict__ part_np /* [block][K][2] */)
 {
-    __shared__ __align__(16) float w0s[kTile];
-    __shared__ __align__(16) float xis[LINEAR ? kTile : 4];
+    // two buffers: the next tile's w_t0 / xi arrive while the rows of this tile stream
+    extern __shared__ __align__(16) float tile_smem[];
+    float (*w0buf)[kTile] = reinterpret_cast<float (*)[kTile]>(tile_smem);
+    float (*xibuf)[kTile] = reinterpret_cast<float (*)[kTile]>(tile_smem + 2 * kTile);   // LINEAR only
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // K < kWarps: warp -> (worker warp % K, share warp / K of nsub); otherwise one warp per worker slot
     const int kc = K < kWarps ? K : kWarps;
@@ -34,25 +47,35 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
 #pragma unroll
     for (int kk = 0; kk < KPW; ++kk) { acc_n[kk] = 0.0; acc_p[kk] = 0.0; }
 
-    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    // park w_t0 / xi of one tile (zeros past the end); asynchronous copies where aligned
+    auto fill = [&](int buf, int64_t tile) {
         const int64_t j0 = tile * kTile;
-        __syncthreads();                                   // the previous tile is no longer read
+        float *w0s = w0buf[buf], *xis = xibuf[buf];
         for (int i = tid * 4; i < kTile; i += kThreads * 4) {
             const int64_t j = j0 + i;
-            float4 b = make_float4(0.f, 0.f, 0.f, 0.f), x = b;
             if (VEC && j + 3 < d) {
-                b = __ldg(reinterpret_cast<const float4 *>(w_t0 + j));
-                if (LINEAR) x = __ldg(reinterpret_cast<const float4 *>(xi + j));
+                cp_async16(w0s + i, w_t0 + j);
+                if (LINEAR) cp_async16(xis + i, xi + j);
             } else {
+                float4 b = make_float4(0.f, 0.f, 0.f, 0.f), x = b;
                 if (j + 0 < d) { b.x = __ldg(w_t0 + j + 0); if (LINEAR) x.x = __ldg(xi + j + 0); }
                 if (j + 1 < d) { b.y = __ldg(w_t0 + j + 1); if (LINEAR) x.y = __ldg(xi + j + 1); }
                 if (j + 2 < d) { b.z = __ldg(w_t0 + j + 2); if (LINEAR) x.z = __ldg(xi + j + 2); }
                 if (j + 3 < d) { b.w = __ldg(w_t0 + j + 3); if (LINEAR) x.w = __ldg(xi + j + 3); }
+                *reinterpret_cast<float4 *>(w0s + i) = b;
+                if (LINEAR) *reinterpret_cast<float4 *>(xis + i) = x;
             }
-            *reinterpret_cast<float4 *>(w0s + i) = b;
-            if (LINEAR) *reinterpret_cast<float4 *>(xis + i) = x;
         }
-        __syncthreads();
+    };
+
+    int buf = 0;
+    if ((int64_t)blockIdx.x < tiles) fill(0, blockIdx.x);
+    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, buf ^= 1) {
+        const int64_t j0 = tile * kTile;
+        cp_async_wait_all();
+        __syncthreads();           // this tile's buffer is complete; the other one is no longer read
+        if (tile + gridDim.x < tiles) fill(buf ^ 1, tile + gridDim.x);
+        const float *w0s = w0buf[buf], *xis = xibuf[buf];
 #pragma unroll
         for (int kk = 0; kk < KPW; ++kk) {
             const int k = wslot + kk * kWarps;
@@ -102,7 +125,7 @@ k_local_state_linear(const float *__restrict__ w, int64_t row_stride, int K, int
         }
         // warps that share a worker add up through shared memory (fixed order)
         __syncthreads();
-        double *red = reinterpret_cast<double *>(w0s);           // [kWarps][2]
+        double *red = reinterpret_cast<double *>(w0buf[0]);      // [kWarps][2]
         if (lane == 0) { red[warp * 2] = n; red[warp * 2 + 1] = pr; }
         __syncthreads();
         const int k = wslot + kk * kWarps;
@@ -143,7 +166,15 @@ template <int KPW>
 cudaError_t launch_kpw(int blocks, bool linear, bool vec, const float *w, int64_t row_stride, int K, int64_t d,
                        const float *w_t0, const float *xi, int64_t tiles, double *part, cudaStream_t s)
 {
-#define FDA_LIN(LI, VE) k_local_state_linear<KPW, LI, VE><<<blocks, kThreads, 0, s>>>(w, row_stride, K, d, w_t0, xi, tiles, part)
+#define FDA_LIN(LI, VE)                                                                            \
+    do {                                                                                           \
+        const int smem = (LI ? 4 : 2) * kTile * (int)sizeof(float);                                \
+        cudaError_t ea = cudaFuncSetAttribute(k_local_state_linear<KPW, LI, VE>,                   \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem);  \
+        if (ea != cudaSuccess) return ea;                                                          \
+        k_local_state_linear<KPW, LI, VE><<<blocks, kThreads, smem, s>>>(w, row_stride, K, d, w_t0, \
+                                                                         xi, tiles, part);         \
+    } while (0)
     if (linear) { if (vec) FDA_LIN(true, true); else FDA_LIN(true, false); }
     else        { if (vec) FDA_LIN(false, true); else FDA_LIN(false, false); }
 #undef FDA_LIN

@@ -646,3 +646,20 @@ def test_repeat_runs_agree_within_tolerance(env):
     b, _ = run_case(env, 8, 50_001, 5, 250, seed=99)
     check_states(b, ref, 5, 250, 50_001)
     assert np.allclose(a, b, rtol=1e-4, atol=1e-7)
+
+
+@pytest.mark.parametrize("n,offset", [(1, 0), (3, 1), (1000, 1), (5_000_003, 3), (1 << 22, 0)])
+def test_read_probe_returns_the_sum(env, n, offset):
+    """The bandwidth probe is not part of the method; its result is the plain sum (fp64 here)."""
+    torch, _, F = env
+    rng = np.random.default_rng(n)
+    x = rng.standard_normal(n + offset).astype(np.float32)
+    buf = torch.from_numpy(x).cuda()
+    out = torch.zeros(1, dtype=torch.float32, device="cuda")
+    with F.FdaContext(0, 0, None, d_max=1024, K_max=1) as ctx:
+        ctx.fda_debug_read_probe(buf[offset:], out)
+        torch.cuda.synchronize()
+        with pytest.raises(F.FdaError):
+            ctx.fda_debug_read_probe(buf[:0], out)
+    want = x[offset:].astype(np.float64).sum()
+    assert abs(float(out.item()) - want) <= 1e-5 * np.abs(x[offset:]).astype(np.float64).sum() + 1e-6
