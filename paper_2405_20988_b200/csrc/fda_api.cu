@@ -98,7 +98,9 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (l > 0 && ctx->columns < 1) { delete ctx; return FDA_ERR_UNSUPPORTED; }
 
     ctx->max_blocks = ctx->n_sm * 4;
-    ctx->tab_stride = (d_max + 63) / 64 * 64;
+    // padded by more than the widest tile of the staged kernel, so that a tile that starts below
+    // d_max never reads past the table (entries past d_max are valid hashes of those indices)
+    ctx->tab_stride = (d_max + 1024 + 63) / 64 * 64;
     ctx->part_sk_floats = l > 0 ? (size_t)ctx->n_sm * ctx->lm * 32 : 0;
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);

@@ -20,9 +20,9 @@ __global__ void k_build_table(const uint64_t *__restrict__ coeffs, int l, uint32
     (void)l;
 }
 
-// 32-bit variant for the staged sketch kernel: bits 0..30 hold the byte offset of the cell in a
-// bins[cell][32] float array, (i*m + bucket) * 128, bit 31 is set when the sign is -1, so that
-// the kernel needs one AND for the address and one AND-XOR for the signed value.
+// 32-bit variant for the staged sketch kernel: bits 0..23 hold the cell i*m + bucket, bit 31 is
+// set when the sign is -1.  The kernel's bins are bins[cell][32] floats, so one shift-and-add
+// (the shift by 7 drops the sign bit) gives the address and one AND-XOR the signed value.
 __global__ void k_build_table32(const uint64_t *__restrict__ coeffs, uint32_t m, uint64_t magic, int64_t n,
                                 int64_t tab_stride, uint32_t *__restrict__ tab)
 {
@@ -33,7 +33,7 @@ __global__ void k_build_table32(const uint64_t *__restrict__ coeffs, uint32_t m,
          j += (int64_t)gridDim.x * blockDim.x) {
         const uint32_t b = fda::bucket_of(c, (uint32_t)j, m, magic);
         const uint32_t s = fda::sign_is_negative(c, (uint32_t)j) ? 0x80000000u : 0u;
-        tab[(size_t)i * tab_stride + j] = (((uint32_t)i * m + b) << 7) | s;
+        tab[(size_t)i * tab_stride + j] = ((uint32_t)i * m + b) | s;
     }
 }
 

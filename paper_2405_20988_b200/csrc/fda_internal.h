@@ -23,7 +23,7 @@ struct fda_ctx {
     // device scratch
     uint64_t *coeffs_dev = nullptr;   // 6*l
     uint16_t *tab = nullptr;          // l planes of tab_stride entries
-    uint32_t *tab32 = nullptr;        // same hash as byte offset | sign<<31 (staged sketch kernel)
+    uint32_t *tab32 = nullptr;        // same hash as cell index | sign<<31 (staged sketch kernel)
     int64_t tab_stride = 0;
     float *part_sk = nullptr;         // per-block sketch partials
     size_t part_sk_floats = 0;

@@ -155,7 +155,7 @@ __device__ __forceinline__ void apply_updates(const uint32_t (&addr)[N], const f
 // quads (eight in flight) or two rows at once (sixteen) were measured slower: what pays is
 // many warps with short windows between load and compare-and-swap, which keeps the share of
 // lost races down.
-template <int LWK, bool LINEAR>
+template <int LWK, bool LINEAR, int ROWS /* sketch rows, 0 = read at run time */>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_w0, const __grid_constant__ CUtensorMap tm_xi,
@@ -211,7 +211,9 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
                                               (uint32_t)(p.rows_per_role * bx) * 4u);
 
     double acc_n = 0.0, acc_p = 0.0;
-    const uint32_t col_addr = bins_addr + (uint32_t)lane * 4u;
+    // table words hold the cell of the whole sketch: take off this role's first cell (the table
+    // is padded past the last tile, so every word read is a valid cell of the row it belongs to)
+    const uint32_t col_addr = bins_addr + (uint32_t)lane * 4u - (((uint32_t)(row0 * p.m)) << 7);
     const int qpb = bx / 4;                                        // quads per box
     const int quads = qpb * nb;                                    // quads per tile
     const int quads_per_pass = ncons * JS * QPL;
@@ -259,23 +261,32 @@ k_local_state_staged(const StagedParams p, const __grid_constant__ CUtensorMap t
             auto row_updates = [&](int i, uint32_t *addr, float *val) {
 #pragma unroll
                 for (int v = 0; v < QPL; ++v) {
-                    // 4 table words of this quad: cell byte offset | sign << 31 (u = 0 where the quad is absent)
+                    // 4 table words of this quad: cell | sign << 31 (u = 0 where the quad is absent)
                     uint32_t h[4];
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(haddr[v] + (uint32_t)(i * bx) * 4u));
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        addr[4 * v + e] = col_addr + (h[e] & 0x7fffffffu);
+                        addr[4 * v + e] = col_addr + (h[e] << 7);     // the shift drops the sign bit
                         val[4 * v + e] = flip(u[4 * v + e], h[e] & 0x80000000u);
                     }
                 }
             };
-            int i = 0;
-            for (; i < rows; ++i) {
-                uint32_t addr[NB];
-                float val[NB];
-                row_updates(i, addr, val);
-                apply_updates<NB>(addr, val);
+            if (ROWS > 0) {
+#pragma unroll
+                for (int i = 0; i < ROWS; ++i) {
+                    uint32_t addr[NB];
+                    float val[NB];
+                    row_updates(i, addr, val);
+                    apply_updates<NB>(addr, val);
+                }
+            } else {
+                for (int i = 0; i < rows; ++i) {
+                    uint32_t addr[NB];
+                    float val[NB];
+                    row_updates(i, addr, val);
+                    apply_updates<NB>(addr, val);
+                }
             }
         }
         acc_n += (double)tile_n;
@@ -443,7 +454,10 @@ template <int LWK>
 cudaError_t launch(fda_ctx *ctx, const StagedParams &p, const CUtensorMap *maps, bool linear, int blocks,
                    int threads, size_t smem, uint32_t flags, float *states, cudaStream_t s)
 {
-    auto kern = linear ? k_local_state_staged<LWK, true> : k_local_state_staged<LWK, false>;
+    // the usual sketch depths get their row loop unrolled
+    auto kern = linear ? k_local_state_staged<LWK, true, 0> : k_local_state_staged<LWK, false, 0>;
+    if (p.roles == 1 && p.l == 5) kern = linear ? k_local_state_staged<LWK, true, 5> : k_local_state_staged<LWK, false, 5>;
+    if (p.roles == 1 && p.l == 7) kern = linear ? k_local_state_staged<LWK, true, 7> : k_local_state_staged<LWK, false, 7>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin);
     if (e != cudaSuccess) return e;
     kern<<<blocks, threads, smem, s>>>(p, maps[0], maps[1], maps[2], maps[3]);
@@ -516,6 +530,8 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
     // Splitting the rows over several blocks was measured slower than the plain-load kernel
     // with fewer bin columns (every role re-stages the tile and amortises it over fewer rows),
     // so this path only takes sketches whose l*m bins fit with 32 columns beside the ring.
+    // (measured again with 372-index tiles and two rows per role at 7 x 500, K = 60: 8.4 ms
+    // against 6.9 ms.)
     if (rows_cap < ctx->l) return cudaErrorNotSupported;
     p.roles = 1;
     p.rows_per_role = ctx->l;
