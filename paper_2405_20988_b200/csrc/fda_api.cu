@@ -46,6 +46,8 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
     cudaFree(ctx->err_flag);
+    cudaFree(ctx->combine_scratch);
+    cudaFree(ctx->combine_ticket);
     cudaFree(ctx->mean_model);
     cudaFree(ctx->stage_w);
     cudaFree(ctx->stage_w_t0);
@@ -115,6 +117,9 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * ctx->part_np_doubles);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->err_flag, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(ctx->err_flag, 0, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_scratch, sizeof(double) * (2 + FDA_MAX_ROWS));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_ticket, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->combine_ticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -40,6 +40,8 @@ struct fda_ctx {
         int K = 0, bx = 0, Kg = 0;
     } tmap_key;
     unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
+    double *combine_scratch = nullptr;        // 2 + FDA_MAX_ROWS doubles: S-bar[0..1] and the row norms
+    unsigned int *combine_ticket = nullptr;   // blocks of the combine kernel that have finished (0 between launches)
     // staging for fda_round_host (lazy)
     float *stage_w = nullptr, *stage_w_t0 = nullptr, *stage_xi = nullptr, *stage_states = nullptr;
     fda_estimate *stage_est = nullptr;
