@@ -368,7 +368,7 @@ def run_ours(args, rank, world, local_rank):
                            "frac_of_peak": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9 / peak,
                            "H": mean_est["H"], "note": "fda_mean_state: S-bar in one pass, no per-worker sketches"},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
-            "roofline": {"kernel": "k_local_state_fast" if args.workload == 4 else "k_local_state_staged", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": {4: "k_local_state_fast", 7: "k_local_state"}.get(args.workload, "k_local_state_staged"), "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "algorithmic_bytes": algo_bytes,
                          "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,

@@ -64,6 +64,12 @@ WORKLOADS = {
                 "heavy", 1e-3, "DenseNet201-sized, 1% of coordinates replaced by 1e-2*t(nu=2)"),
     5: Workload("convnextlarge", 197_767_336, 8, 5, 250, 0.06, (1e-2,), 4, "iid", 1e-4,
                 "ConvNeXt-Large-sized, iid drift"),
+    # a second shape (Table 2: VGG16* with 2.6M parameters; Section 3.3 leaves other sketch
+    # sizes open): the recommended sketch and a larger one
+    6: Workload("vgg16star", 2_600_000, 20, 5, 250, 0.06, (1e-2,), 11, "shared", 1e-3,
+                "VGG16*-sized, shared + private drift"),
+    7: Workload("vgg16star-8x1000", 2_600_000, 20, 8, 1000, 0.06 * (250.0 / 1000.0) ** 0.5, (1e-2,), 11,
+                "shared", 1e-3, "VGG16*-sized, shared + private drift, 8 x 1000 sketch"),
 }
 
 SHARED_SIGMA = 5e-4
