@@ -224,7 +224,19 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         if dist:
             dist.barrier()
+        late = False
+        if not sampler.lines:
+            # the timed region was shorter than one sampling period: keep the same load running
+            # (untimed) until the sampler has seen it
+            late = True
+            t_end = time.perf_counter() + 1.5
+            while len(sampler.lines) < 2 and time.perf_counter() < t_end:
+                for _ in range(20):
+                    step(False)
+                torch.cuda.synchronize()
         clocks = sampler.stop()
+        if late:
+            clocks["sampled"] = "under the same load right after the timed steps (they took less than one sample period)"
         parts = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in evs])
         return parts, clocks
 
