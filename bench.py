@@ -43,7 +43,7 @@ SMEM_CAS_UPDATES_PER_CLK_SM = 6.8     # measured on B200: bare fp32 shared-memor
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
 # capture summarised under profiles/ (None: not captured for the kernel as it stands).
-LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: 5_164_300_000, 5: 11_076_300_000}
+LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: 5_165_200_000, 5: 11_079_400_000}
 
 
 def measured_hbm_peak():
