@@ -107,7 +107,9 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
-        if (e == cudaSuccess && (size_t)ctx->lm * 128 < ((size_t)1 << 31))
+        // the 32-bit table serves the staged sketch kernel only, which needs all l*m bins with 32
+        // columns plus its ring in shared memory
+        if (e == cudaSuccess && (size_t)ctx->lm * 128 + 16384 <= (size_t)ctx->smem_optin)
             e = cudaMalloc(&ctx->tab32, sizeof(uint32_t) * (size_t)l * ctx->tab_stride);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
         if (e == cudaSuccess)

@@ -663,3 +663,38 @@ def test_read_probe_returns_the_sum(env, n, offset):
             ctx.fda_debug_read_probe(buf[:0], out)
     want = x[offset:].astype(np.float64).sum()
     assert abs(float(out.item()) - want) <= 1e-5 * np.abs(x[offset:]).astype(np.float64).sum() + 1e-6
+
+
+def test_one_context_serves_changing_shapes_and_buffers(env):
+    """A context created for (d_max, K_max) is then called with smaller and different shapes and
+    with fresh buffers; state that the library keeps between calls (cached tensor maps, partial
+    buffers, the combine ticket) must not leak from one call into the next."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(2024)
+    l, m = 5, 250
+    coeffs = rand_coeffs(rng, l)
+    shapes = [(8, 33_001), (5, 4_099), (8, 33_001), (16, 50_000), (3, 777), (8, 33_001)]
+    keep = []                                  # keep earlier buffers alive: new calls get new addresses
+    with F.FdaContext(l, m, coeffs, d_max=50_000, K_max=16) as ctx:
+        buf = ctx.new_estimate_buffer()
+        for K, d in shapes:
+            stride = S.row_stride(d)
+            w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+            wbuf = np.zeros((K, stride), dtype=np.float32)
+            wbuf[:, :d] = w_t0 + rng.normal(0, 1e-3, size=(K, d)).astype(np.float32)
+            xi = rng.normal(size=d)
+            xi = (xi / np.linalg.norm(xi)).astype(np.float32)
+            w, w0, xg, st = gpu_states(torch, F, ctx, wbuf, w_t0, xi)
+            keep.append((w, w0, xg, st))
+            for _ in range(2):                 # the second call reuses the cached tensor maps
+                st.fill_(float("nan"))
+                ctx.fda_local_state(w[:, :d], w0, xg, ALL, st)
+                torch.cuda.synchronize()
+                got = st.cpu().numpy()
+                ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, l, m)
+                check_states(got, ora, l, m, d)
+            for variant in (0, 1):
+                ref = oracle.combine(got, l, m, variant, 0.06, 1e-3)
+                e = ctx.fda_combine_estimate(st, K, variant, np.float32(0.06), 1e-3, buf).as_dict()
+                tol = check_estimate(e, ref, l)
+                check_trigger(e, ref, 1e-3, tol)
