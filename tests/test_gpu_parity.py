@@ -698,3 +698,75 @@ def test_one_context_serves_changing_shapes_and_buffers(env):
                 e = ctx.fda_combine_estimate(st, K, variant, np.float32(0.06), 1e-3, buf).as_dict()
                 tol = check_estimate(e, ref, l)
                 check_trigger(e, ref, 1e-3, tol)
+
+
+def _random_case(seed):
+    """Seeded random shape: worker count, dimension, sketch size, alignment, pitch, flags."""
+    rng = np.random.default_rng(10_000 + seed)
+    K = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 48, 64, 70]))
+    d = int(rng.choice([1, 2, 5, 31, 127, 128, 129, 1000, 4095, 4096, 4097, 9973, 20_011, 40_009]))
+    l, m = [(5, 250), (7, 500), (1, 1), (2, 3), (3, 64), (4, 251), (6, 400), (8, 333), (16, 100), (5, 1000)][
+        int(rng.integers(0, 10))]
+    misalign = int(rng.choice([0, 0, 0, 1, 2, 3]))
+    stride = S.row_stride(d) + int(rng.choice([0, 0, 1, 4, 32]))
+    flags = int(rng.choice([7, 7, 7, 5, 4, 6, 3]))
+    sigma = float(rng.choice([1e-4, 1e-3, 1e-1]))
+    return K, d, l, m, misalign, stride, flags, sigma
+
+
+@pytest.mark.parametrize("seed", range(36))
+def test_local_state_random_shapes(env, seed):
+    K, d, l, m, misalign, stride, flags, sigma = _random_case(seed)
+    run_case(env, K, d, l, m, seed=seed, flags=flags, misalign=misalign, stride=stride, sigma=sigma)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_whole_round_random_shapes(env, seed):
+    """Random shape, whole round: states -> estimate (both variants, a threshold on either side
+    of the oracle's H) -> gated average with direction refresh -> states after the sync are zero."""
+    torch, oracle, F = env
+    K, d, l, m, misalign, stride, _, sigma = _random_case(100 + seed)
+    rng = np.random.default_rng(500 + seed)
+    coeffs = rand_coeffs(rng, l)
+    w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+    wbuf = np.zeros((K, stride), dtype=np.float32)
+    shared = rng.normal(0, 0.5 * sigma, size=d)
+    wbuf[:, :d] = w_t0 + (shared + rng.normal(0, sigma, size=(K, d))).astype(np.float32)
+    xi = rng.normal(size=d)
+    xi = (xi / np.linalg.norm(xi)).astype(np.float32)
+    ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, l, m)
+    eps = 0.06
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        w, w0, xg, st = gpu_states(torch, F, ctx, wbuf, w_t0, xi, ALL, misalign)
+        buf = ctx.new_estimate_buffer()
+        ctx.fda_local_state(w[:, :d], w0, xg, ALL, st)
+        torch.cuda.synchronize()
+        got = st.cpu().numpy()
+        check_states(got, ora, l, m, d)
+        ms = torch.full((ctx.state_len,), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.fda_mean_state(w[:, :d], w0, xg, ALL, ms)
+        torch.cuda.synchronize()
+        ubar = (wbuf[:, :d].astype(np.float64) - w_t0.astype(np.float64)).mean(axis=0)
+        check_mean_state(ms.cpu().numpy(), ora, float(ubar @ ubar), l, m, d, K)
+        fired = None
+        for variant in (0, 1):
+            h = oracle.combine(got, l, m, variant, eps, 0.0)["H"]
+            for theta in (abs(h) * 2.0 + 1e-30, abs(h) * 0.5):
+                ref = oracle.combine(got, l, m, variant, eps, theta)
+                e = ctx.fda_combine_estimate(st, K, variant, np.float32(eps), np.float32(theta), buf).as_dict()
+                tol = check_estimate(e, ref, l)
+                check_trigger(e, ref, theta, tol)
+                fired = bool(e["trigger"])
+        ref_avg = oracle.average(wbuf[:, :d])
+        xi_new = torch.full((d + 4,), 9.0, dtype=torch.float32, device="cuda")[misalign:misalign + d]
+        ctx.fda_average_models_xi(w[:, :d], w0, xi_new, buf, F.FDA_AVG_BROADCAST)
+        torch.cuda.synchronize()
+        if fired:
+            check_average(w0.cpu().numpy(), ref_avg)
+            assert all(np.array_equal(w.cpu().numpy()[k, :d], w0.cpu().numpy()) for k in range(K))
+            ctx.fda_local_state(w[:, :d], w0, xi_new, ALL, st)
+            torch.cuda.synchronize()
+            assert not st.cpu().numpy().any()              # all drifts are zero after the sync
+        else:
+            assert np.array_equal(w0.cpu().numpy(), w_t0)
+            assert bool((xi_new == 9.0).all())
