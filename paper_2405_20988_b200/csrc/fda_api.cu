@@ -43,6 +43,8 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->coeffs_dev);
     cudaFree(ctx->tab);
     cudaFree(ctx->tab32);
+    cudaFree(ctx->sched);
+    cudaFree(ctx->sched_used);
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
     cudaFree(ctx->err_flag);
@@ -123,6 +125,7 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_ticket, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(ctx->combine_ticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
+    if (e == cudaSuccess) e = fda_build_gather_schedule(ctx, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         const fda_status st = e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;

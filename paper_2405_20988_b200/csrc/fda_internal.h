@@ -11,6 +11,21 @@
 // Hash-table entry: bits 0..14 bucket, bit 15 set when the sign is -1.
 #define FDA_TAB_SIGN_BIT 0x8000u
 
+// Geometry of the sorted-list sketch kernel (fda_local_state_gather.cu) and of its schedule
+// (fda_sched.cu).  A tile is nbox boxes of kGatherBox indices; entries address rows of the
+// transposed drift tile: bits 0..12 row, bit 15 set when the sign is -1.
+constexpr int kGatherWorkers = 8;      // workers per group (one 32-byte row of the drift tile)
+constexpr int kGatherBox = 256;        // indices per tensor box (rows of 1 KB: whole 128-byte lines)
+constexpr int kGatherSlots = 16;       // lists walked side by side by one warp
+constexpr int kGatherMaxLen = 32;      // longest list of one slot (longer cells are split)
+constexpr int kGatherPrefixBytes = 2304; // shared memory in front of the schedule headers (scalars, fp64 sums)
+constexpr int kGatherPadRows = 4;      // zero rows behind the tile, one per 32-byte bank group
+
+// byte offset of the cell ids inside a schedule record with room for nr_max rounds
+inline __host__ __device__ int fda_sched_cells_off(int nr_max) { return ((2 + 2 * nr_max) * 2 + 15) / 16 * 16; }
+// bytes of one ring stage of the sketch kernel: a [workers][box] tile of w, a box of w_t0, a box of xi
+inline int fda_gather_stage_bytes() { return kGatherWorkers * kGatherBox * 4 + 2 * kGatherBox * 4; }
+
 struct fda_ctx {
     int device = 0;
     int n_sm = 0;
@@ -30,6 +45,15 @@ struct fda_ctx {
     double *part_np = nullptr;        // per-block (norm, projection) partials
     size_t part_np_doubles = 0;
     int max_blocks = 0;
+    // gather schedule of the sorted-list sketch kernel (null when not built)
+    unsigned char *sched = nullptr;   // [tile][row] records of sched_pitch bytes
+    size_t sched_pitch = 0;
+    uint16_t *sched_used = nullptr;   // [tile][row] 128-byte entry chunks a record uses
+    int sched_nbox = 0;               // boxes of kGatherBox indices per tile
+    int sched_nr_max = 0;             // rounds a record has room for
+    int sched_hdr_bytes = 0;          // bytes of a record's header (round table + cell ids)
+    int sched_max_chunks = 0;         // 128-byte entry chunks a record has room for
+    int64_t sched_tiles = 0;
     float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
     // tensor maps of the last staged launch (encoding four maps costs several microseconds of
     // host time, which matters for small models); valid while the key below matches
@@ -60,6 +84,10 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s);
 cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, cudaStream_t s);
+cudaError_t fda_build_gather_schedule(fda_ctx *ctx, cudaStream_t s);   // allocates and fills ctx->sched when it fits
+cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);
 cudaError_t fda_launch_local_state_linear(fda_ctx *ctx, const float *w, int64_t row_stride, int K,

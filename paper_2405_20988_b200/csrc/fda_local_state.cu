@@ -466,7 +466,9 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
                                    float *states, cudaStream_t s)
 {
     {   // aligned sketch requests take the bulk-copy staged kernel
-        cudaError_t e = fda_launch_local_state_staged(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
+        cudaError_t e = fda_launch_local_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
+        if (e != cudaErrorNotSupported) return e;
+        e = fda_launch_local_state_staged(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
         if (e != cudaErrorNotSupported) return e;
         e = fda_launch_local_state_linear(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
         if (e != cudaErrorNotSupported) return e;
