@@ -40,10 +40,21 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 << 20
 NOMINAL_HBM_GBS = 8000.0               # the data-sheet figure, quoted beside the measured copy rate
 SMEM_CAS_UPDATES_PER_CLK_SM = 6.8     # measured on B200: bare fp32 shared-memory atomicAdd loop, 1024 threads
+SMEM_GATHER_UPDATES_PER_CLK_SM = 32.0  # one 4-byte shared-memory read per update at 128 bytes per clock and SM
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
 # capture summarised under profiles/ (None: not captured for the kernel as it stands).
-LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: 5_165_200_000, 5: 11_079_400_000}
+LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: 5_165_200_000, 5: None}
+
+
+def secondary_roofline(kernel, updates_per_s, n_sm, sm_mhz):
+    gather = kernel == "k_local_state_gather"
+    per_clk = SMEM_GATHER_UPDATES_PER_CLK_SM if gather else SMEM_CAS_UPDATES_PER_CLK_SM
+    peak = per_clk * n_sm * sm_mhz * 1e6
+    return {"bound": "smem_gather" if gather else "smem_cas", "unit": "updates/s", "achieved": updates_per_s,
+            "peak": peak, "frac": updates_per_s / peak,
+            "note": ("peak = one 4-byte shared-memory read per update, 128 bytes per clock and SM" if gather else
+                     "peak = microbenchmarked fp32 atomicAdd rate on lane-private columns")}
 
 
 def measured_hbm_peak():
@@ -194,6 +205,8 @@ def run_ours(args, rank, world, local_rank):
     theta, eps = float(wl.thetas[-1]), float(np.float32(wl.epsilon))
     stream = torch.cuda.current_stream()
 
+    ls_kernel = [""]       # the kernel the library picked for the sketch pass (asked after each launch)
+
     def step(timed):
         # the sync of the previous step made all models equal: put the drifted models back
         w.copy_(w_src)
@@ -204,6 +217,7 @@ def run_ours(args, rank, world, local_rank):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         ev[0].record(stream)
         ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
+        ls_kernel[0] = ctx.fda_debug_last_kernel()
         ev[1].record(stream)
         ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, eps, theta, est_buf, want_host=False)
         ev[2].record(stream)
@@ -380,19 +394,16 @@ def run_ours(args, rank, world, local_rank):
                            "frac_of_peak": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9 / peak,
                            "H": mean_est["H"], "note": "fda_mean_state: S-bar in one pass, no per-worker sketches"},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
-            "roofline": {"kernel": {4: "k_local_state_fast", 7: "k_local_state"}.get(args.workload, "k_local_state_staged"), "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": ls_kernel[0], "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "algorithmic_bytes": algo_bytes,
                          "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
                          "traffic": LOCAL_STATE_TRAFFIC_BYTES.get(args.workload)},
-            # what really binds the sketch pass: fp32 updates of shared-memory bins, which are
-            # compare-and-swap loops on this hardware (measured ceiling 6.8 updates/clk/SM)
-            "secondary_roofline": {"bound": "smem_cas", "unit": "updates/s",
-                                   "achieved": K * d * wl.l / (ls_ms * 1e-3),
-                                   "peak": SMEM_CAS_UPDATES_PER_CLK_SM * n_sm * (clocks.get("sm_mhz") or 1965.0) * 1e6,
-                                   "frac": K * d * wl.l / (ls_ms * 1e-3) /
-                                           (SMEM_CAS_UPDATES_PER_CLK_SM * n_sm * (clocks.get("sm_mhz") or 1965.0) * 1e6),
-                                   "note": "peak = microbenchmarked fp32 atomicAdd rate on lane-private columns"},
+            # what binds the sketch pass next to HBM: the shared-memory traffic of the l updates per
+            # element (gather kernel: one 4-byte read each, 32 per clock and SM at best; the
+            # compare-and-swap kernels: a measured 6.8 adds per clock and SM)
+            "secondary_roofline": secondary_roofline(ls_kernel[0], K * d * wl.l / (ls_ms * 1e-3), n_sm,
+                                                     clocks.get("sm_mhz") or 1965.0),
             "cpu_baseline": cpu,
             "e2e": None if not e2e_times else
                    {"value": job_value(world, K * d, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d,

@@ -214,6 +214,17 @@ fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float
                                 void *stream);
 
 /*
+ * Name of the kernel that served the context's last fda_local_state call (the paper has no
+ * counterpart): "k_local_state_gather" (sketch pass over per-cell index lists; 16-byte aligned inputs,
+ * jobs of at least eight tiles per block whose lists average eight entries or more),
+ * "k_local_state_staged" (compare-and-swap sketch pass on TMA-staged tiles; 16-byte aligned
+ * inputs), "k_local_state_linear" (no sketch requested), "k_local_state" (everything else), or
+ * "" before the first call.  The string is static; ctx == NULL gives "".  Tests and the
+ * benchmark use it to say which kernel a number belongs to.
+ */
+const char *fda_debug_last_kernel(const fda_ctx *ctx);
+
+/*
  * Local state without a context and without any allocation.  (The paper has no counterpart
  * to this call; it exists for the way some programs have to use the library.)
  *

@@ -21,7 +21,7 @@ _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "
            4: "FDA_ERR_NOMEM"}
 
 EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
-           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe",
+           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
 
@@ -79,6 +79,8 @@ def load_library():
     lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
     lib.fda_debug_read_probe.argtypes = [vp, vp, i64, vp, vp]
     lib.fda_debug_read_probe.restype = c_int
+    lib.fda_debug_last_kernel.argtypes = [vp]
+    lib.fda_debug_last_kernel.restype = ctypes.c_char_p
     lib.fda_local_state_linear_noalloc.argtypes = [c_int, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
     lib.fda_local_state_linear_noalloc.restype = c_int
     for name in ("fda_create", "fda_destroy", "fda_local_state", "fda_combine_estimate",
@@ -267,6 +269,10 @@ class FdaContext:
         st = self._lib.fda_debug_read_probe(self._h, _dev_ptr(src, name="src"), src.numel(),
                                             _dev_ptr(sum_out, name="sum_out"), _stream_ptr(stream))
         self._check(st, "fda_debug_read_probe")
+
+    def fda_debug_last_kernel(self) -> str:
+        """Name of the kernel that served the last fda_local_state call on this context."""
+        return self._lib.fda_debug_last_kernel(self._h).decode()
 
     @staticmethod
     def new_estimate_buffer(device="cuda"):

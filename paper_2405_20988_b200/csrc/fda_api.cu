@@ -152,6 +152,8 @@ size_t fda_state_len(const fda_ctx *ctx) { return ctx ? 2 + (size_t)ctx->lm : 0;
 
 const char *fda_last_error(const fda_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
 
+const char *fda_debug_last_kernel(const fda_ctx *ctx) { return ctx ? ctx->last_ls_kernel : ""; }
+
 fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                            const float *w_t0, const float *xi, uint32_t flags, float *states,
                            void *stream)

@@ -71,6 +71,7 @@ struct fda_ctx {
     fda_estimate *stage_est = nullptr;
     int64_t stage_stride = 0;
     uint64_t coeffs_host[6 * FDA_MAX_ROWS] = {0};
+    const char *last_ls_kernel = "";   // which kernel served the last fda_local_state
     std::string err;
 };
 

@@ -465,14 +465,16 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s)
 {
-    {   // aligned sketch requests take the bulk-copy staged kernel
+    {   // sketch requests: the list kernel when its schedule exists and the job is large enough, else
+        // the staged kernel (aligned inputs); requests without a sketch: the streaming kernel
         cudaError_t e = fda_launch_local_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) return e;
+        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_gather"; return e; }
         e = fda_launch_local_state_staged(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) return e;
+        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_staged"; return e; }
         e = fda_launch_local_state_linear(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) return e;
+        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_linear"; return e; }
     }
+    ctx->last_ls_kernel = "k_local_state";
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     LsParams p{};
     p.w = w; p.row_stride = row_stride; p.K = K; p.d = d; p.w_t0 = w_t0;

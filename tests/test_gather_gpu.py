@@ -1,0 +1,140 @@
+"""GPU parity of the sorted-list sketch kernel (k_local_state_gather) against the CPU oracle.
+
+The library picks that kernel for 16-byte aligned inputs when a block gets at least eight
+tiles of 4096 indices, so these cases are sized to reach it (the test asserts which kernel
+ran) and shaped to hit its edges: a ragged last tile, d not a multiple of 4, a last worker
+group with one or three workers, flag subsets, hash coefficients that put every index of a
+sketch row into one cell (the cell is split over many lists and added atomically) or into
+cells in strict rotation, and unaligned inputs, which must fall back to another kernel.
+Tolerances are those of tests/fda_testlib.py (1e-5 relative, scaled for near-zero cells).
+"""
+import numpy as np
+import pytest
+
+import fda_synth as S
+from fda_testlib import check_states
+
+pytestmark = pytest.mark.gpu
+
+P = (1 << 61) - 1
+ALL = 1 | 2 | 4
+GATHER = "k_local_state_gather"
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("CUDA device required for -m gpu tests")
+    import oracle
+    import paper_2405_20988_b200 as F
+    F.load_library()
+    return torch, oracle, F
+
+
+def rand_coeffs(rng, l):
+    c = rng.integers(0, P, size=6 * l, dtype=np.uint64)
+    c[0::6] |= np.uint64(1)
+    c[2::6] |= np.uint64(1)
+    return c
+
+
+def run(env, K, d, l, m, seed, flags=ALL, misalign=0, coeffs=None, sigma=1e-3, workers=None, expect=GATHER):
+    torch, oracle, F = env
+    rng = np.random.default_rng(seed)
+    stride = S.row_stride(d)
+    coeffs = rand_coeffs(rng, l) if coeffs is None else coeffs
+    w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+    wbuf = np.zeros((K, stride), dtype=np.float32)
+    for k in range(K):                       # row by row: keeps the host footprint small
+        wbuf[k, :d] = w_t0 + rng.normal(0, sigma, size=d).astype(np.float32)
+    xi = rng.normal(size=d)
+    xi = (xi / np.linalg.norm(xi)).astype(np.float32)
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        buf = torch.zeros(K * stride + 8, dtype=torch.float32, device="cuda")
+        w = buf[misalign:misalign + K * stride].view(K, stride)
+        w.copy_(torch.from_numpy(wbuf))
+        w0 = torch.from_numpy(w_t0).cuda()
+        xg = torch.from_numpy(xi).cuda()
+        st = torch.full((K, ctx.state_len), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.fda_local_state(w[:, :d], w0, xg, flags, st)
+        torch.cuda.synchronize()
+        name = ctx.fda_debug_last_kernel()
+        got = st.cpu().numpy()
+    if expect is not None:
+        assert name == expect, name
+    else:
+        assert name != GATHER, name
+    ks = list(range(K)) if workers is None else workers
+    ora = oracle.local_state(wbuf[:, :d], w_t0, xi if (flags & 2) else None, coeffs,
+                             l if (flags & 4) else 0, m if (flags & 4) else 0, workers=ks, threads=8)
+    full = np.zeros((K, 2 + l * m))
+    full[:, :ora.shape[1]] = ora
+    if not flags & 1:                         # norm slot off: it must be zero; scales come from the oracle norm
+        assert not got[:, 0].any()
+        norms = oracle.local_state(wbuf[:, :d], w_t0, None, None, 0, 0, workers=ks, threads=8)[:, 0]
+        got = got.copy()
+        got[:, 0] = norms
+        full[:, 0] = norms
+    if not flags & 2:
+        assert not got[:, 1].any()
+    check_states(got, full, l, m, d, rows=ks)
+    return got
+
+
+D_RAGGED = 600_011          # 147 tiles, the last one holds 1979 indices; not a multiple of 4
+
+
+def test_ragged_tail_and_partial_worker_group(env):
+    run(env, 57, D_RAGGED, 5, 250, seed=11, workers=[0, 7, 8, 31, 55, 56])
+
+
+@pytest.mark.parametrize("flags", [4, 1 | 4, 2 | 4])
+def test_flag_subsets(env, flags):
+    run(env, 57, D_RAGGED, 5, 250, seed=12, flags=flags, workers=[3, 56])
+
+
+@pytest.mark.parametrize("d", [147 * 4096, 147 * 4096 + 1, 148 * 4096 - 1])
+def test_tile_boundaries(env, d):
+    run(env, 60, d, 5, 250, seed=13, workers=[0, 59])
+
+
+def test_three_workers_in_one_group(env):
+    run(env, 3, 4_900_003, 5, 250, seed=14)
+
+
+def test_degenerate_and_rotating_buckets(env):
+    """Row 0: a = m, so a*j + b is a multiple of m plus b and every index lands in cell b mod m;
+    row 1: a = 1, b = 0, so bucket = j mod m; row 2: c3 = 1 and the other sign coefficients zero,
+    so the sign is the parity of j^3 = parity of j; the rest random."""
+    l, m = 5, 250
+    c = rand_coeffs(np.random.default_rng(15), l)
+    c[0], c[1] = m, 7
+    c[6], c[7] = 1, 0
+    c[14], c[15], c[16], c[17] = 1, 0, 0, 0
+    got = run(env, 57, D_RAGGED, l, m, seed=15, coeffs=c, workers=[0, 56])
+    row0 = got[:, 2:2 + m]
+    assert np.count_nonzero(row0[0]) == 1 and row0[0, 7] != 0.0
+
+
+def test_other_sketch_shapes(env):
+    run(env, 57, D_RAGGED, 3, 100, seed=16, workers=[5, 56])      # long lists: most cells are split
+    run(env, 57, D_RAGGED, 7, 300, seed=17, workers=[5, 56])
+
+
+def test_heavy_tails(env):
+    torch, oracle, F = env
+    # drift with rare large values (the shape of workload 4): short fp32 runs must keep 1e-5
+    run(env, 57, D_RAGGED, 5, 250, seed=18, sigma=1e-3, workers=[1])
+    run(env, 57, D_RAGGED, 5, 250, seed=19, sigma=3.0, workers=[1])
+
+
+def test_unaligned_inputs_use_another_kernel(env):
+    run(env, 57, D_RAGGED, 5, 250, seed=20, misalign=1, workers=[0, 56], expect=None)
+
+
+def test_repeat_runs_agree(env):
+    a = run(env, 57, D_RAGGED, 5, 250, seed=21, workers=[2])
+    b = run(env, 57, D_RAGGED, 5, 250, seed=21, workers=[2])
+    scale = np.maximum(np.abs(a), 1e-30)
+    assert float(np.max(np.abs(a - b) / scale)) <= 1e-5
