@@ -12,15 +12,22 @@
 // and SM against 6 for compare-and-swap adds into the bins.
 //
 // A block serves a group of up to 8 workers and a strided set of tiles.  Per tile:
-//   phase 1  the tile arrives as [8 workers][256 indices] tensor boxes (TMA ring,
-//            zero fill outside the tensor, no multicast); 16 warps subtract w_t0, add up
-//            ||u||^2 and <xi,u>, and store u transposed: ut[index][worker], 32 bytes per index;
-//   phase 2  all warps draw (round, sketch row) items from a counter, load the item's entries
-//            from the schedule (prefetched into L2 during phase 1), gather and flush.
+//   phase 1  16 loader warps bring the tile in with 16-byte asynchronous copies, 512 indices of
+//            the 8 workers per step, each warp into its own part of a small ring (it reads back
+//            only what it copied itself, so the ring needs no barrier, only the warp's own copy
+//            groups); they subtract w_t0, add up ||u||^2 and <xi,u>, and store u transposed:
+//            ut[index][worker], 32 bytes per index.  One more warp fetches the schedule headers
+//            of the next tile and prefetches this tile's entries into L2;
+//   phase 2  all 32 warps walk the lists: item (round r, sketch row i) goes to warp
+//            (r*l + i) mod 32; the warp loads the item's entries, gathers and adds the 16 sums
+//            to the bins.
 // Lane = (slot q, half h): slot q walks one list, the two halves hold workers 4h .. 4h+3, so a
 // gather is one 128-bit load per lane and a quarter-warp reads four 32-byte rows.
-// Every wait on a barrier is bounded: when it runs out the thread raises the context's error
-// word and stops waiting, so the kernel always returns.
+// The phases are separated by __syncthreads; nothing in this kernel waits on another block or
+// on a barrier object.  Measured on B200 while this was built: tensor copies (TMA) of
+// [8][252] or [8][256] boxes into a ring delivered 8-11 bytes per clock and SM here, no better
+// than these copies; staging the tile in registers with scalar coalesced loads was slower
+// (0.62 against 0.44 ms at d = 20M, K = 8).
 
 #include <algorithm>
 
