@@ -43,7 +43,7 @@ constexpr uint32_t kPrefix = kGatherPrefixBytes;   // counters and the warps' (n
 constexpr int kSlab = 2 * kGatherBox;          // indices staged per step: 32 per loader warp
 constexpr uint32_t kUnitBytes = 1280;          // one warp's part of a stage: W [8][32], W0 [32], XI [32]
 constexpr int kMaxStages = 6;                  // slab stages of the ring (copy groups pending per thread)
-constexpr int kMaxChunks = kGatherMaxLen / 4;  // entry chunks of one round
+static_assert(kGatherMaxLen == 32, "walk_item is instantiated for up to 8 chunks of four steps");
 static_assert(kLoaderWarps * 32 == kSlab, "a slab is 32 indices per loader warp");
 static_assert(kLoaderWarps * (int)kUnitBytes == 2 * (kGatherWorkers * kGatherBox * 4 + 2 * kGatherBox * 4),
               "ring stage size differs from the one the tile size was chosen with");
@@ -66,12 +66,6 @@ struct GatherParams {
     double *part_np;                 // [block][GW][2]
 };
 
-__device__ __forceinline__ float4 lds128(uint32_t addr)
-{
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ float lds32(uint32_t addr)
 {
     float v;
@@ -82,21 +76,47 @@ __device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c,
 {
     asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
-// acc += s * v for two packed fp32 pairs (s = +1 or -1: exact)
-__device__ __forceinline__ void fma2(float &a0, float &a1, float v0, float v1, float s)
+// Two schedule entries (the halves of one 32-bit word): gather the two rows and add them with
+// their signs.  The sums stay packed as fp32 pairs from the first step to the flush, the loaded
+// row arrives as two 64-bit registers, and the sign is a multiplication by (+-1, +-1) (exact),
+// so a step is: one field extract, one address, one load, sign word, pair, two packed FMAs.
+__device__ __forceinline__ void gather_pair(uint32_t w, uint32_t lane_base, unsigned long long &a01,
+                                            unsigned long long &a23)
 {
-    asm("{\n\t.reg .b64 a, v, ss;\n\t"
-        "mov.b64 a, {%0,%1};\n\tmov.b64 v, {%2,%3};\n\tmov.b64 ss, {%4,%4};\n\t"
-        "fma.rn.f32x2 a, v, ss, a;\n\tmov.b64 {%0,%1}, a;\n\t}"
-        : "+f"(a0), "+f"(a1) : "f"(v0), "f"(v1), "f"(s));
+    uint32_t r1;
+    asm("bfe.u32 %0, %1, 16, 13;" : "=r"(r1) : "r"(w));
+    const uint32_t ad0 = lane_base + ((w & 0x1fffu) << 5), ad1 = lane_base + (r1 << 5);
+    unsigned long long u0, u1, v0, v1, ss0, ss1;
+    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(u0), "=l"(u1) : "r"(ad0));
+    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(v0), "=l"(v1) : "r"(ad1));
+    const uint32_t s0 = ((w << 16) & 0x80000000u) ^ 0x3f800000u;      // bit 15: sign of the low entry
+    const uint32_t s1 = (w & 0x80000000u) ^ 0x3f800000u;              // bit 31: sign of the high entry
+    asm("mov.b64 %0, {%1,%1};" : "=l"(ss0) : "r"(s0));
+    asm("mov.b64 %0, {%1,%1};" : "=l"(ss1) : "r"(s1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a01) : "l"(u0), "l"(ss0));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a23) : "l"(u1), "l"(ss0));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a01) : "l"(v0), "l"(ss1));
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a23) : "l"(v1), "l"(ss1));
 }
-// one schedule entry: gather the row, add it with the entry's sign
-__device__ __forceinline__ void gather_step(uint32_t e, uint32_t lane_base, float4 &acc)
+
+// One item: NCH chunks of four steps for this lane's slot (the last chunk holds two or four;
+// `steps` is even).  All loads of the entries first, then the walk.
+template <int NCH>
+__device__ __forceinline__ float4 walk_item(const uint2 *ent, int steps, uint32_t lane_base)
 {
-    const float4 v = lds128(lane_base + ((e & 0x1fffu) << 5));
-    const float s = __uint_as_float(0x3f800000u ^ ((e & 0x8000u) << 16));
-    fma2(acc.x, acc.y, v.x, v.y, s);
-    fma2(acc.z, acc.w, v.z, v.w, s);
+    uint2 ch[NCH];
+#pragma unroll
+    for (int cc = 0; cc < NCH; ++cc) ch[cc] = __ldg(ent + cc * kGatherSlots);
+    unsigned long long a01 = 0ull, a23 = 0ull;
+#pragma unroll
+    for (int cc = 0; cc < NCH; ++cc) {
+        gather_pair(ch[cc].x, lane_base, a01, a23);
+        if (cc + 1 < NCH || 4 * NCH - 2 < steps) gather_pair(ch[cc].y, lane_base, a01, a23);
+    }
+    float4 acc;
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.x), "=f"(acc.y) : "l"(a01));
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.z), "=f"(acc.w) : "l"(a23));
+    return acc;
 }
 
 // 16-byte asynchronous copy global -> shared; bytes past `src_bytes` (0..16) arrive as zero
@@ -299,21 +319,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const Gather
                 const uint32_t cell = reinterpret_cast<const uint16_t *>(hrow + fda_sched_cells_off(p.nr_max))[r * kGatherSlots + q];
                 const uint2 *ent = reinterpret_cast<const uint2 *>(rec0 + (size_t)i * p.pitch + p.hdr_bytes +
                                                                    (size_t)coff * 128) + q;
-                uint2 ch[kMaxChunks];
-#pragma unroll
-                for (int cc = 0; cc < kMaxChunks; ++cc)
-                    if (4 * cc < steps) ch[cc] = __ldg(ent + cc * kGatherSlots);
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int cc = 0; cc < kMaxChunks; ++cc) {
-                    if (4 * cc < steps) {                       // steps is even
-                        gather_step(ch[cc].x & 0xffffu, gather_base, acc);
-                        gather_step(ch[cc].x >> 16, gather_base, acc);
-                    }
-                    if (4 * cc + 2 < steps) {
-                        gather_step(ch[cc].y & 0xffffu, gather_base, acc);
-                        gather_step(ch[cc].y >> 16, gather_base, acc);
-                    }
+                float4 acc;
+                switch ((steps + 3) >> 2) {                     // straight-line code per chunk count
+                    case 1: acc = walk_item<1>(ent, steps, gather_base); break;
+                    case 2: acc = walk_item<2>(ent, steps, gather_base); break;
+                    case 3: acc = walk_item<3>(ent, steps, gather_base); break;
+                    case 4: acc = walk_item<4>(ent, steps, gather_base); break;
+                    case 5: acc = walk_item<5>(ent, steps, gather_base); break;
+                    case 6: acc = walk_item<6>(ent, steps, gather_base); break;
+                    case 7: acc = walk_item<7>(ent, steps, gather_base); break;
+                    default: acc = walk_item<8>(ent, steps, gather_base); break;
                 }
                 float *b = bins + (cell & 0x7fffu) * GW + h * 4;
                 if (cell & 0x8000u) {                           // a cell with several lists
