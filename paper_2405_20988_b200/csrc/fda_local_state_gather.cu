@@ -358,40 +358,48 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const Gather
     }
 }
 
-// states[k][.] = sum of the partials of worker k's blocks, in block order, in fp64.
+// states[k][.] = sum of the partials of worker k's blocks in fp64, in a fixed order: four
+// adjacent lanes share one output, lane s adds the blocks s, s + 4, ... of the worker's group in
+// order (eight loads in flight), and the four sums are added as (s0 + s1) + (s2 + s3).
 __global__ void k_finalize_gather(const GatherParams p, int blocks, uint32_t flags, float *__restrict__ states)
 {
     const int lm = p.l * p.m, slen = 2 + lm;
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
-    const int64_t total = (int64_t)p.groups * slen * GW;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+    const int64_t total = (int64_t)p.groups * slen * GW * 4;
+    const int64_t padded = (total + 31) & ~(int64_t)31;                 // whole warps take part in the shuffles
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < padded;
          t += (int64_t)gridDim.x * blockDim.x) {
-        const int kl = (int)(t % GW);
-        const int e = (int)((t / GW) % slen);
-        const int g = (int)(t / ((int64_t)GW * slen));
+        const bool valid = t < total;
+        const int sub = (int)(t & 3);
+        const int64_t o = t >> 2;
+        const int kl = (int)(o % GW);
+        const int e = (int)((o / GW) % slen);
+        const int g = (int)(o / ((int64_t)GW * slen));
         const int k = g * GW + kl;
-        if (k >= p.K) continue;
+        const int nb = (blocks - g + p.groups - 1) / p.groups;        // blocks of this group: g, g + groups, ...
         double acc = 0.0;
-        if (e < 2) {
+        if (!valid) {
+        } else if (e < 2) {
             const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0
                                      : ((flags & FDA_STATE_LINEAR) != 0 && p.have_xi);
             if (on)
-                for (int b = g; b < blocks; b += p.groups) acc += p.part_np[((size_t)b * GW + kl) * 2 + e];
+                for (int j = sub; j < nb; j += 4) acc += p.part_np[((size_t)(g + j * p.groups) * GW + kl) * 2 + e];
         } else if (sketch) {
-            const size_t pitch = (size_t)lm * GW;
-            const float *src = p.part_sk + (size_t)g * pitch + (size_t)(e - 2) * GW + kl;
-            const size_t step = pitch * p.groups;
-            int b = g;
-            for (; b + 7 * p.groups < blocks; b += 8 * p.groups, src += 8 * step) {     // eight loads in flight, added in block order
+            const size_t step = (size_t)lm * GW * p.groups;             // from one block of the group to the next
+            const float *src = p.part_sk + (size_t)g * lm * GW + (size_t)(e - 2) * GW + kl + (size_t)sub * step;
+            int j = sub;
+            for (; j + 28 < nb; j += 32, src += 32 * step) {
                 float v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = src[u * step];
+                for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(4 * u) * step];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) acc += (double)v[u];
             }
-            for (; b < blocks; b += p.groups, src += step) acc += (double)src[0];
+            for (; j < nb; j += 4, src += 4 * step) acc += (double)src[0];
         }
-        states[(size_t)k * slen + e] = (float)acc;
+        const double pair = acc + __shfl_xor_sync(0xffffffffu, acc, 1);      // lanes 0,1: s0 + s1; lanes 2,3: s2 + s3
+        const double other = __shfl_xor_sync(0xffffffffu, pair, 2);
+        if (valid && sub == 0 && k < p.K) states[(size_t)k * slen + e] = (float)(pair + other);
     }
 }
 
@@ -444,7 +452,7 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     kern<<<blocks, kThreads, smem, s>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int64_t total = (int64_t)p.groups * (2 + ctx->lm) * GW;
+    const int64_t total = (int64_t)p.groups * (2 + ctx->lm) * GW * 4;
     int fb = (int)((total + 255) / 256);
     if (fb > ctx->n_sm * 8) fb = ctx->n_sm * 8;
     k_finalize_gather<<<fb, 256, 0, s>>>(p, blocks, flags, states);

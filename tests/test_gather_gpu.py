@@ -138,3 +138,23 @@ def test_repeat_runs_agree(env):
     b = run(env, 57, D_RAGGED, 5, 250, seed=21, workers=[2])
     scale = np.maximum(np.abs(a), 1e-30)
     assert float(np.max(np.abs(a - b) / scale)) <= 1e-5
+
+
+def test_last_kernel_names_follow_the_dispatch(env):
+    """Small jobs and jobs without a sketch are served by the other kernels, and the library says so."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(22)
+    d, K, l, m = 50_000, 4, 5, 250
+    coeffs = rand_coeffs(rng, l)
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        assert ctx.fda_debug_last_kernel() == ""
+        w = torch.randn((K, d), device="cuda")
+        w0 = torch.randn(d, device="cuda")
+        st = torch.empty((K, ctx.state_len), device="cuda")
+        ctx.fda_local_state(w, w0, None, 1 | 4, st)
+        assert ctx.fda_debug_last_kernel() == "k_local_state_staged"
+        ctx.fda_local_state(w, w0, None, 1, st)
+        assert ctx.fda_debug_last_kernel() == "k_local_state_linear"
+        ctx.fda_local_state(w[:, 1:], w0[1:], None, 1 | 4, st)          # rows start at an odd element
+        assert ctx.fda_debug_last_kernel() == "k_local_state"
+        torch.cuda.synchronize()
