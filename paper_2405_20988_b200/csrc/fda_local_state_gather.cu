@@ -66,16 +66,6 @@ struct GatherParams {
     double *part_np;                 // [block][GW][2]
 };
 
-__device__ __forceinline__ float lds32(uint32_t addr)
-{
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d)
-{
-    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 // Two schedule entries (the halves of one 32-bit word): gather the two rows and add them with
 // their signs.  The sums stay packed as fp32 pairs from the first step to the flush, the loaded
 // row arrives as two 64-bit registers, and the sign is a multiplication by (+-1, +-1) (exact),
@@ -237,29 +227,32 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const Gather
                 load_slab();                     // the slab S-1 ahead, into the stage read last time
                 cp_async_wait(S - 1);            // this thread's copies of the slab to read have landed
                 __syncwarp();                    // ... and so have the other lanes'
-                const uint32_t src = my_ring + (uint32_t)rd_stage * slab_stage_bytes;
+                const float *src = reinterpret_cast<const float *>(smem_raw + ring_off + (uint32_t)warp * kUnitBytes +
+                                                                   (uint32_t)rd_stage * slab_stage_bytes);
                 if (++rd_stage == S) rd_stage = 0;
                 // two steps: lanes h = 0 take index q with workers 4*hh .. 4*hh+3, lanes h = 1 index
                 // 16 + q with the other four (rows of the unit are 32 floats: the halves use
-                // different banks); the second step swaps the worker halves
+                // different banks); the second step swaps the worker halves.  All ten loads first.
+                const int xl = 16 * h + q;
+                const float w0 = src[256 + xl];
+                const float xv = LINEAR ? src[288 + xl] : 0.f;
+                float wv[2][4];
+#pragma unroll
+                for (int step = 0; step < 2; ++step)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) wv[step][e] = src[(4 * (h ^ step) + e) * 32 + xl];
 #pragma unroll
                 for (int step = 0; step < 2; ++step) {
                     const int hh = h ^ step;
-                    const int xl = 16 * h + q;
-                    const uint32_t wa = src + (uint32_t)((4 * hh) * 32 + xl) * 4u;
-                    const float w0 = lds32(src + 1024u + (uint32_t)xl * 4u);
-                    const float u0 = lds32(wa) - w0;
-                    const float u1 = lds32(wa + 128u) - w0;
-                    const float u2 = lds32(wa + 256u) - w0;
-                    const float u3 = lds32(wa + 384u) - w0;
+                    const float u0 = wv[step][0] - w0, u1 = wv[step][1] - w0, u2 = wv[step][2] - w0, u3 = wv[step][3] - w0;
                     nf[step][0] = fmaf(u0, u0, nf[step][0]); nf[step][1] = fmaf(u1, u1, nf[step][1]);
                     nf[step][2] = fmaf(u2, u2, nf[step][2]); nf[step][3] = fmaf(u3, u3, nf[step][3]);
                     if (LINEAR) {
-                        const float xv = lds32(src + 1152u + (uint32_t)xl * 4u);
                         pf[step][0] = fmaf(xv, u0, pf[step][0]); pf[step][1] = fmaf(xv, u1, pf[step][1]);
                         pf[step][2] = fmaf(xv, u2, pf[step][2]); pf[step][3] = fmaf(xv, u3, pf[step][3]);
                     }
-                    sts128(ut_addr + (uint32_t)(sb * kSlab + 32 * warp + xl) * 32u + (uint32_t)hh * 16u, u0, u1, u2, u3);
+                    *reinterpret_cast<float4 *>(ut + (size_t)(sb * kSlab + 32 * warp + xl) * GW + 4 * hh) =
+                        make_float4(u0, u1, u2, u3);
                 }
                 __syncwarp();                    // all reads of this stage are done before it is refilled
             }
