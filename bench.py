@@ -44,7 +44,7 @@ SMEM_GATHER_UPDATES_PER_CLK_SM = 32.0  # one 4-byte shared-memory read per updat
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
 # capture summarised under profiles/ (None: not captured for the kernel as it stands).
-LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: 950_300_000, 4: 5_165_200_000, 5: 9_581_300_000}
+LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: 949_400_000, 4: 5_165_200_000, 5: 9_579_100_000}
 
 
 def secondary_roofline(kernel, updates_per_s, n_sm, sm_mhz):

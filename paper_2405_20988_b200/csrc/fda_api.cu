@@ -109,13 +109,21 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
+        // the list schedule first: where it exists the staged kernel only serves jobs of fewer than
+        // eight tiles per block, and its table need not cover more indices than those
+        if (e == cudaSuccess) e = fda_build_gather_schedule(ctx, nullptr);
+        ctx->tab32_stride = ctx->tab_stride;
+        if (ctx->sched) {
+            const int64_t cap = ((int64_t)8 * ctx->n_sm * ctx->sched_nbox * kGatherBox + 1024 + 63) / 64 * 64;
+            if (cap < ctx->tab32_stride) ctx->tab32_stride = cap;
+        }
         // the 32-bit table serves the staged sketch kernel only, which needs all l*m bins with 32
         // columns plus its ring in shared memory
         if (e == cudaSuccess && (size_t)ctx->lm * 128 + 16384 <= (size_t)ctx->smem_optin)
-            e = cudaMalloc(&ctx->tab32, sizeof(uint32_t) * (size_t)l * ctx->tab_stride);
+            e = cudaMalloc(&ctx->tab32, sizeof(uint32_t) * (size_t)l * ctx->tab32_stride);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
-        if (e == cudaSuccess)
-            e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
     }
     ctx->part_np_doubles = (size_t)ctx->max_blocks * (size_t)(K_max > 32 ? K_max : 32) * 2;
     if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * ctx->part_np_doubles);
@@ -125,7 +133,6 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_ticket, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(ctx->combine_ticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
-    if (e == cudaSuccess) e = fda_build_gather_schedule(ctx, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         const fda_status st = e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;

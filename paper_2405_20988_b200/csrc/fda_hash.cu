@@ -69,9 +69,11 @@ cudaError_t fda_launch_build_table(const fda_ctx *ctx, cudaStream_t s)
     dim3 grid(blocks_for(ctx->tab_stride, 256, ctx->n_sm * 16), (unsigned)ctx->l);
     k_build_table<<<grid, 256, 0, s>>>(ctx->coeffs_dev, ctx->l, (uint32_t)ctx->m, magic,
                                       ctx->tab_stride, ctx->tab_stride, ctx->tab);
-    if (ctx->tab32)
-        k_build_table32<<<grid, 256, 0, s>>>(ctx->coeffs_dev, (uint32_t)ctx->m, magic, ctx->tab_stride,
-                                            ctx->tab_stride, ctx->tab32);
+    if (ctx->tab32) {
+        dim3 grid32(blocks_for(ctx->tab32_stride, 256, ctx->n_sm * 16), (unsigned)ctx->l);
+        k_build_table32<<<grid32, 256, 0, s>>>(ctx->coeffs_dev, (uint32_t)ctx->m, magic, ctx->tab32_stride,
+                                              ctx->tab32_stride, ctx->tab32);
+    }
     return cudaGetLastError();
 }
 

@@ -40,6 +40,7 @@ struct fda_ctx {
     uint16_t *tab = nullptr;          // l planes of tab_stride entries
     uint32_t *tab32 = nullptr;        // same hash as cell index | sign<<31 (staged sketch kernel)
     int64_t tab_stride = 0;
+    int64_t tab32_stride = 0;         // entries per plane of tab32: the indices the staged kernel may be asked for
     float *part_sk = nullptr;         // per-block sketch partials
     size_t part_sk_floats = 0;
     double *part_np = nullptr;        // per-block (norm, projection) partials

@@ -479,6 +479,7 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
                                           uint32_t flags, float *states, cudaStream_t s)
 {
     if (!(flags & FDA_STATE_SKETCH) || ctx->l == 0 || !ctx->tab32) return cudaErrorNotSupported;
+    if (d + 1024 > ctx->tab32_stride) return cudaErrorNotSupported;      // the table covers smaller jobs only
     const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
     const bool aligned = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) &&
                          (row_stride % 4 == 0);
@@ -582,8 +583,8 @@ cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t 
                            (uint64_t)row_stride * 4, (uint32_t)bx, (uint32_t)p.Kg);
         ok = ok && make_map(&maps[1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, w_t0, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
         ok = ok && make_map(&maps[2], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, xi_key, (uint64_t)d, 1, vec_pitch, (uint32_t)bx, 1);
-        ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT32, ctx->tab32, (uint64_t)ctx->tab_stride,
-                            (uint64_t)ctx->l, (uint64_t)ctx->tab_stride * 4, (uint32_t)bx, (uint32_t)p.rows_per_role);
+        ok = ok && make_map(&maps[3], CU_TENSOR_MAP_DATA_TYPE_UINT32, ctx->tab32, (uint64_t)ctx->tab32_stride,
+                            (uint64_t)ctx->l, (uint64_t)ctx->tab32_stride * 4, (uint32_t)bx, (uint32_t)p.rows_per_role);
         if (!ok) return cudaErrorNotSupported;
         key.w = w; key.w_t0 = w_t0; key.xi = xi_key; key.row_stride = row_stride; key.d = d;
         key.K = K; key.bx = bx; key.Kg = p.Kg;
