@@ -214,6 +214,23 @@ fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float
                                 void *stream);
 
 /*
+ * Copy of one record of the list schedule that k_local_state_gather walks (the paper has no
+ * counterpart; Section 3.1 only fixes what the sketch sums).  The record of (tile, row) lists the
+ * tile's indices cell by cell: 16-bit words [0] rounds, [2 .. 2+NR) steps of round r,
+ * [2+NR .. 2+2NR) first 128-byte chunk of round r; from byte cells_offset on cells[r][16] (cell
+ * index row*m + bucket, bit 15 set when the cell has several lists, l*m for an unused slot); from
+ * byte header_bytes on chunks [slot][4] of entries, entry = index inside the tile (bits 0..12, or
+ * tile_indices + 0..3 for padding) | sign << 15, steps 4c .. 4c+3 of the round.
+ * record_host: host buffer of `capacity` bytes, receives min(capacity, record_bytes) bytes.
+ * info (host, 8 values): tile_indices, NR, header_bytes, record_bytes, slots (16), longest list
+ * (32), cells_offset, tiles in the schedule.  Synchronises the device.
+ * Errors: INVALID_ARG (NULL, tile or row out of range), UNSUPPORTED (the context has no schedule:
+ * no sketch, lists too short for it, or not enough free memory at fda_create), CUDA.
+ */
+fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, int row, void *record_host,
+                              size_t capacity, int64_t *info);
+
+/*
  * Name of the kernel that served the context's last fda_local_state call (the paper has no
  * counterpart): "k_local_state_gather" (sketch pass over per-cell index lists; 16-byte aligned inputs,
  * jobs of at least eight tiles per block whose lists average eight entries or more),

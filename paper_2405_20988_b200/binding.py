@@ -21,7 +21,7 @@ _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "
            4: "FDA_ERR_NOMEM"}
 
 EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
-           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel",
+           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel", "fda_debug_schedule",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
 
@@ -79,6 +79,8 @@ def load_library():
     lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
     lib.fda_debug_read_probe.argtypes = [vp, vp, i64, vp, vp]
     lib.fda_debug_read_probe.restype = c_int
+    lib.fda_debug_schedule.argtypes = [vp, i64, c_int, vp, ctypes.c_size_t, vp]
+    lib.fda_debug_schedule.restype = c_int
     lib.fda_debug_last_kernel.argtypes = [vp]
     lib.fda_debug_last_kernel.restype = ctypes.c_char_p
     lib.fda_local_state_linear_noalloc.argtypes = [c_int, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
@@ -269,6 +271,18 @@ class FdaContext:
         st = self._lib.fda_debug_read_probe(self._h, _dev_ptr(src, name="src"), src.numel(),
                                             _dev_ptr(sum_out, name="sum_out"), _stream_ptr(stream))
         self._check(st, "fda_debug_read_probe")
+
+    def fda_debug_schedule(self, tile: int, row: int):
+        """(record bytes as a numpy uint8 array, info dict) of the list schedule's record (tile, row)."""
+        info = (ctypes.c_int64 * 8)()
+        probe = (ctypes.c_uint8 * 16)()
+        st = self._lib.fda_debug_schedule(self._h, tile, row, probe, 16, info)
+        self._check(st, "fda_debug_schedule")
+        buf = np.zeros(int(info[3]), dtype=np.uint8)
+        st = self._lib.fda_debug_schedule(self._h, tile, row, buf.ctypes.data_as(ctypes.c_void_p), buf.size, info)
+        self._check(st, "fda_debug_schedule")
+        keys = ("tile_indices", "nr_max", "header_bytes", "record_bytes", "slots", "max_len", "cells_offset", "tiles")
+        return buf, dict(zip(keys, (int(v) for v in info)))
 
     def fda_debug_last_kernel(self) -> str:
         """Name of the kernel that served the last fda_local_state call on this context."""

@@ -353,6 +353,31 @@ fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets
     return FDA_OK;
 }
 
+fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, int row, void *record_host,
+                              size_t capacity, int64_t *info)
+{
+    if (!ctx || !record_host || !info) return FDA_ERR_INVALID_ARG;
+    if (!ctx->sched) return FDA_ERR_UNSUPPORTED;
+    if (tile < 0 || tile >= ctx->sched_tiles || row < 0 || row >= ctx->l) return FDA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FDA_ERR_CUDA;
+    info[0] = (int64_t)ctx->sched_nbox * kGatherBox;
+    info[1] = ctx->sched_nr_max;
+    info[2] = ctx->sched_hdr_bytes;
+    info[3] = (int64_t)ctx->sched_pitch;
+    info[4] = kGatherSlots;
+    info[5] = kGatherMaxLen;
+    info[6] = fda_sched_cells_off(ctx->sched_nr_max);
+    info[7] = ctx->sched_tiles;
+    const size_t n = capacity < ctx->sched_pitch ? capacity : ctx->sched_pitch;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess)
+        e = cudaMemcpy(record_host, ctx->sched + ((size_t)tile * ctx->l + row) * ctx->sched_pitch, n,
+                       cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }
+    return FDA_OK;
+}
+
 fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float *sum_out, void *stream)
 {
     if (!ctx) return FDA_ERR_INVALID_ARG;
