@@ -110,7 +110,9 @@ const char *fda_last_error(const fda_ctx *ctx);
  *   states      out, K x state_len floats
  * Any alignment of w, w_t0, xi is accepted; 16-byte aligned pointers with row_stride a
  * multiple of 4 take the vector path.  Errors: INVALID_ARG (NULL, K < 1 or > K_max, d < 1
- * or > d_max, row_stride < d, unknown flag, SKETCH without a sketch), CUDA.
+ * or > d_max, row_stride < d, unknown flag, SKETCH without a sketch), UNSUPPORTED (more worker
+ * groups than the context's partial-sum scratch holds: K above 4 x the SM count with a list
+ * schedule, above 32 x the SM count without; nothing is launched), CUDA.
  */
 fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                            const float *w_t0, const float *xi, uint32_t flags, float *states,
@@ -215,20 +217,28 @@ fda_status fda_debug_read_probe(fda_ctx *ctx, const float *src, int64_t n, float
 
 /*
  * Copy of one record of the list schedule that k_local_state_gather walks (the paper has no
- * counterpart; Section 3.1 only fixes what the sketch sums).  The record of (tile, row) lists the
- * tile's indices cell by cell: 16-bit words [0] rounds, [2 .. 2+NR) steps of round r,
- * [2+NR .. 2+2NR) first 128-byte chunk of round r; from byte cells_offset on cells[r][16] (cell
- * index row*m + bucket, bit 15 set when the cell has several lists, l*m for an unused slot); from
- * byte header_bytes on chunks [slot][4] of entries, entry = index inside the tile (bits 0..12, or
- * tile_indices + 0..3 for padding) | sign << 15, steps 4c .. 4c+3 of the round.
+ * counterpart; Section 3.1 only fixes what the sketch sums).  The record of a tile lists the
+ * tile's indices cell by cell for every sketch row.  Layout (byte offsets):
+ *   [0] u32 items  [4] u32 bytes of the record  [8] u32 entry chunks  [12] u32 0
+ *   [16] items x { u16 steps, u16 cell block, u32 first chunk }, most steps first
+ *   cells_offset = 16 + 8*items rounded up to 64: cell blocks of 32 u16, the cell index
+ *       row*m + bucket of the list a lane walks (bit 15 set when the cell has several lists,
+ *       l*m when the lane has none)
+ *   entries_offset = cells_offset + 64*items rounded up to 256: chunks of 256 bytes,
+ *       chunk[lane][4] u16 entries for steps 4c .. 4c+3 of an item; entry = row of the drift
+ *       tile (bits 0..12) | sign << 15, where index r of the tile is stored in row
+ *       r ^ ((r >> 3) & 3) and rows tile_indices + r, r < 8, are padding (zeros).
+ * In every step the eight lanes 8q .. 8q+7 of an item address rows in eight different 16-byte
+ * bank groups (row mod 8), so that the shared-memory load of the step is conflict free.
  * record_host: host buffer of `capacity` bytes, receives min(capacity, record_bytes) bytes.
- * info (host, 8 values): tile_indices, NR, header_bytes, record_bytes, slots (16), longest list
- * (32), cells_offset, tiles in the schedule.  Synchronises the device.
- * Errors: INVALID_ARG (NULL, tile or row out of range), UNSUPPORTED (the context has no schedule:
+ * info (host, 8 values): tile_indices, lanes per item (32), longest list (64), record_bytes,
+ * tiles in the schedule, padding rows (8), lanes per pass (8), bytes of the whole schedule.
+ * Synchronises the device.
+ * Errors: INVALID_ARG (NULL, tile out of range), UNSUPPORTED (the context has no schedule:
  * no sketch, lists too short for it, or not enough free memory at fda_create), CUDA.
  */
-fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, int row, void *record_host,
-                              size_t capacity, int64_t *info);
+fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_host, size_t capacity,
+                              int64_t *info);
 
 /*
  * Name of the kernel that served the context's last fda_local_state call (the paper has no

@@ -79,7 +79,7 @@ def load_library():
     lib.fda_debug_hash.argtypes = [vp, i64, i64, vp, vp, vp]
     lib.fda_debug_read_probe.argtypes = [vp, vp, i64, vp, vp]
     lib.fda_debug_read_probe.restype = c_int
-    lib.fda_debug_schedule.argtypes = [vp, i64, c_int, vp, ctypes.c_size_t, vp]
+    lib.fda_debug_schedule.argtypes = [vp, i64, vp, ctypes.c_size_t, vp]
     lib.fda_debug_schedule.restype = c_int
     lib.fda_debug_last_kernel.argtypes = [vp]
     lib.fda_debug_last_kernel.restype = ctypes.c_char_p
@@ -272,16 +272,17 @@ class FdaContext:
                                             _dev_ptr(sum_out, name="sum_out"), _stream_ptr(stream))
         self._check(st, "fda_debug_read_probe")
 
-    def fda_debug_schedule(self, tile: int, row: int):
-        """(record bytes as a numpy uint8 array, info dict) of the list schedule's record (tile, row)."""
+    def fda_debug_schedule(self, tile: int):
+        """(record bytes as a numpy uint8 array, info dict) of the list schedule's record of a tile."""
         info = (ctypes.c_int64 * 8)()
         probe = (ctypes.c_uint8 * 16)()
-        st = self._lib.fda_debug_schedule(self._h, tile, row, probe, 16, info)
+        st = self._lib.fda_debug_schedule(self._h, tile, probe, 16, info)
         self._check(st, "fda_debug_schedule")
         buf = np.zeros(int(info[3]), dtype=np.uint8)
-        st = self._lib.fda_debug_schedule(self._h, tile, row, buf.ctypes.data_as(ctypes.c_void_p), buf.size, info)
+        st = self._lib.fda_debug_schedule(self._h, tile, buf.ctypes.data_as(ctypes.c_void_p), buf.size, info)
         self._check(st, "fda_debug_schedule")
-        keys = ("tile_indices", "nr_max", "header_bytes", "record_bytes", "slots", "max_len", "cells_offset", "tiles")
+        keys = ("tile_indices", "slots", "max_len", "record_bytes", "tiles", "pad_rows", "lanes_per_pass",
+                "schedule_bytes")
         return buf, dict(zip(keys, (int(v) for v in info)))
 
     def fda_debug_last_kernel(self) -> str:

@@ -35,6 +35,7 @@ fda_status fail_cuda(fda_ctx *ctx, cudaError_t e, const char *where)
     if (ctx) {
         ctx->err = std::string(where) + ": " + cudaGetErrorString(e);
     }
+    if (e == cudaErrorNotSupported) return FDA_ERR_UNSUPPORTED;      // a launcher refused the shape
     return e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;
 }
 
@@ -44,7 +45,7 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->tab);
     cudaFree(ctx->tab32);
     cudaFree(ctx->sched);
-    cudaFree(ctx->sched_used);
+    cudaFree(ctx->sched_off);
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
     cudaFree(ctx->err_flag);
@@ -113,10 +114,10 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
             e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
         // the list schedule first: where it exists the staged kernel only serves jobs of fewer than
         // eight tiles per block, and its table need not cover more indices than those
-        if (e == cudaSuccess) e = fda_build_gather_schedule(ctx, nullptr);
+        if (e == cudaSuccess) e = fda_build_list_schedule(ctx, nullptr);
         ctx->tab32_stride = ctx->tab_stride;
         if (ctx->sched) {
-            const int64_t cap = ((int64_t)8 * ctx->n_sm * ctx->sched_nbox * kGatherBox + 1024 + 63) / 64 * 64;
+            const int64_t cap = ((int64_t)8 * ctx->n_sm * ctx->sched_T + 1024 + 63) / 64 * 64;
             if (cap < ctx->tab32_stride) ctx->tab32_stride = cap;
         }
         // the 32-bit table serves the staged sketch kernel only, which needs all l*m bins with 32
@@ -353,27 +354,28 @@ fda_status fda_debug_hash(fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets
     return FDA_OK;
 }
 
-fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, int row, void *record_host,
-                              size_t capacity, int64_t *info)
+fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_host, size_t capacity,
+                              int64_t *info)
 {
     if (!ctx || !record_host || !info) return FDA_ERR_INVALID_ARG;
     if (!ctx->sched) return FDA_ERR_UNSUPPORTED;
-    if (tile < 0 || tile >= ctx->sched_tiles || row < 0 || row >= ctx->l) return FDA_ERR_INVALID_ARG;
+    if (tile < 0 || tile >= ctx->sched_tiles) return FDA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FDA_ERR_CUDA;
-    info[0] = (int64_t)ctx->sched_nbox * kGatherBox;
-    info[1] = ctx->sched_nr_max;
-    info[2] = ctx->sched_hdr_bytes;
-    info[3] = (int64_t)ctx->sched_pitch;
-    info[4] = kGatherSlots;
-    info[5] = kGatherMaxLen;
-    info[6] = fda_sched_cells_off(ctx->sched_nr_max);
-    info[7] = ctx->sched_tiles;
-    const size_t n = capacity < ctx->sched_pitch ? capacity : ctx->sched_pitch;
+    uint64_t off[2] = {0, 0};
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess)
-        e = cudaMemcpy(record_host, ctx->sched + ((size_t)tile * ctx->l + row) * ctx->sched_pitch, n,
-                       cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(off, ctx->sched_off + tile, sizeof(off), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }
+    info[0] = ctx->sched_T;
+    info[1] = kListSlots;
+    info[2] = kListMaxLen;
+    info[3] = (int64_t)(off[1] - off[0]);
+    info[4] = ctx->sched_tiles;
+    info[5] = kListPadRows;
+    info[6] = kListOct;
+    info[7] = (int64_t)ctx->sched_bytes;
+    const size_t n = capacity < (size_t)info[3] ? capacity : (size_t)info[3];
+    e = cudaMemcpy(record_host, ctx->sched + off[0], n, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }
     return FDA_OK;
 }

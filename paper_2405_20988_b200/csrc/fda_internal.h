@@ -12,19 +12,31 @@
 #define FDA_TAB_SIGN_BIT 0x8000u
 
 // Geometry of the sorted-list sketch kernel (fda_local_state_gather.cu) and of its schedule
-// (fda_sched.cu).  A tile is nbox boxes of kGatherBox indices; entries address rows of the
-// transposed drift tile: bits 0..12 row, bit 15 set when the sign is -1.
-constexpr int kGatherWorkers = 8;      // workers per group (one 32-byte row of the drift tile)
-constexpr int kGatherBox = 256;        // indices per tensor box (rows of 1 KB: whole 128-byte lines)
-constexpr int kGatherSlots = 16;       // lists walked side by side by one warp
-constexpr int kGatherMaxLen = 32;      // longest list of one slot (longer cells are split)
-constexpr int kGatherPrefixBytes = 2304; // shared memory in front of the schedule headers (scalars, fp64 sums)
-constexpr int kGatherPadRows = 4;      // zero rows behind the tile, one per 32-byte bank group
+// (fda_sched.cu).  Entries address rows of the drift tile ut[index][4 workers]: bits 0..12 row,
+// bit 15 set when the sign is -1.  Index r of a tile lives in row r ^ ((r >> 3) & 3).
+constexpr int kListWorkers = 4;        // workers per group: one 16-byte row of the drift tile
+constexpr int kListSlots = 32;         // lists walked side by side by one warp (lane = list)
+constexpr int kListOct = 8;            // lanes per pass of a 128-bit shared-memory load = 16-byte bank groups
+constexpr int kListMaxLen = 64;        // longest list (longer cells are cut into pieces)
+constexpr int kListPadRows = 8;        // zero rows behind the tile, one per bank group
+constexpr int kListBatch = 1024;       // indices a producer step covers; tiles are multiples of it
+constexpr int kListMaxTile = 7168;     // rows + pad rows must fit 13 bits
+constexpr int kListMinTilesPerBlock = 1;
 
-// byte offset of the cell ids inside a schedule record with room for nr_max rounds
-inline __host__ __device__ int fda_sched_cells_off(int nr_max) { return ((2 + 2 * nr_max) * 2 + 15) / 16 * 16; }
-// bytes of one ring stage of the sketch kernel: a [workers][box] tile of w, a box of w_t0, a box of xi
-inline int fda_gather_stage_bytes() { return kGatherWorkers * kGatherBox * 4 + 2 * kGatherBox * 4; }
+// byte offsets inside the schedule record of a tile with `items` items
+inline __host__ __device__ size_t fda_sched_cells_off(uint32_t items) { return ((size_t)16 + 8 * (size_t)items + 63) / 64 * 64; }
+inline __host__ __device__ size_t fda_sched_entries_off(uint32_t items)
+{
+    return (fda_sched_cells_off(items) + (size_t)items * kListSlots * 2 + 255) / 256 * 256;
+}
+// shared memory of the sketch kernel: one item-table buffer; everything for a tile of T indices
+inline __host__ __device__ uint32_t fda_list_row(uint32_t r) { return r ^ ((r >> 3) & 3u); }
+inline int fda_list_table_bytes(int ni_max) { return (16 + 8 * ni_max + 15) / 16 * 16; }
+inline size_t fda_list_smem_bytes(int l, int m, int T, int ni_max)
+{
+    return 576 + 2 * (size_t)fda_list_table_bytes(ni_max) + (size_t)l * m * kListWorkers * 4 +
+           2 * (size_t)(T + kListPadRows) * kListWorkers * 4;
+}
 
 struct fda_ctx {
     int device = 0;
@@ -46,15 +58,16 @@ struct fda_ctx {
     double *part_np = nullptr;        // per-block (norm, projection) partials
     size_t part_np_doubles = 0;
     int max_blocks = 0;
-    // gather schedule of the sorted-list sketch kernel (null when not built)
-    unsigned char *sched = nullptr;   // [tile][row] records of sched_pitch bytes
-    size_t sched_pitch = 0;
-    uint16_t *sched_used = nullptr;   // [tile][row] 128-byte entry chunks a record uses
-    int sched_nbox = 0;               // boxes of kGatherBox indices per tile
-    int sched_nr_max = 0;             // rounds a record has room for
-    int sched_hdr_bytes = 0;          // bytes of a record's header (round table + cell ids)
-    int sched_max_chunks = 0;         // 128-byte entry chunks a record has room for
+    // list schedule of the sorted-list sketch kernel (null when not built)
+    unsigned char *sched = nullptr;   // records of the tiles, 256-byte aligned
+    uint64_t *sched_off = nullptr;    // [tiles + 1] byte offsets of the records
+    uint64_t sched_bytes = 0;         // size of the schedule
+    uint64_t sched_skipped_bytes = 0; // size of a schedule that was not kept (memory limit)
+    int64_t sched_limit_bytes = 0;    // caller's cap on the schedule (0: a third of the free memory)
+    int sched_T = 0;                  // indices per tile
+    int sched_ni_max = 0;             // items a record can have
     int64_t sched_tiles = 0;
+    double sched_build_ms = 0.0;      // host time spent building it
     float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
     // tensor maps of the last staged launch (encoding four maps costs several microseconds of
     // host time, which matters for small models); valid while the key below matches
@@ -88,7 +101,7 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
 cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);
-cudaError_t fda_build_gather_schedule(fda_ctx *ctx, cudaStream_t s);   // allocates and fills ctx->sched when it fits
+cudaError_t fda_build_list_schedule(fda_ctx *ctx, cudaStream_t s);   // allocates and fills ctx->sched when it fits
 cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);

@@ -507,6 +507,12 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
     if ((int64_t)groups * cpg > ctx->max_blocks) cpg = ctx->max_blocks / groups;
     p.cpg = (int)cpg;
     const int blocks = groups * p.cpg;
+    // the partial sums of a launch must fit the context's scratch (sized for n_sm blocks of 32
+    // worker lanes and 4 * n_sm blocks of K_max workers): more worker groups than that is refused
+    if (blocks < 1 || (sketch && (size_t)blocks * p.lm * lwk > ctx->part_sk_floats) ||
+        (size_t)blocks * lwk * 2 > ctx->part_np_doubles)
+        return cudaErrorNotSupported;
+    ctx->last_ls_kernel = fast ? "k_local_state_fast" : "k_local_state";
 
     size_t smem = (size_t)(threads / 32) * lwk * 2 * sizeof(double);
     if (sketch) {

@@ -1,11 +1,10 @@
 """GPU parity of the sorted-list sketch kernel (k_local_state_gather) against the CPU oracle.
 
-The library picks that kernel for 16-byte aligned inputs when a block gets at least eight
-tiles of 4096 indices, so these cases are sized to reach it (the test asserts which kernel
-ran) and shaped to hit its edges: a ragged last tile, d not a multiple of 4, a last worker
-group with one or three workers, flag subsets, hash coefficients that put every index of a
-sketch row into one cell (the cell is split over many lists and added atomically) or into
-cells in strict rotation, and unaligned inputs, which must fall back to another kernel.
+The library picks that kernel whenever the context holds a list schedule (the test asserts
+which kernel ran); the cases are shaped to hit its edges: a ragged last tile, d not a multiple of
+4, a last worker group with one or three workers, flag subsets, hash coefficients that put every
+index of a sketch row into one cell (the cell is cut into many lists and added atomically) or into
+cells in strict rotation, and rows that are only 4-byte aligned (32-bit loads).
 Tolerances are those of tests/fda_testlib.py (1e-5 relative, scaled for near-zero cells).
 """
 import numpy as np
@@ -82,7 +81,7 @@ def run(env, K, d, l, m, seed, flags=ALL, misalign=0, coeffs=None, sigma=1e-3, w
     return got
 
 
-D_RAGGED = 600_011          # 147 tiles, the last one holds 1979 indices; not a multiple of 4
+D_RAGGED = 600_011          # 98 tiles of 6144 indices, the last one holds 4043; not a multiple of 4
 
 
 def test_ragged_tail_and_partial_worker_group(env):
@@ -94,7 +93,7 @@ def test_flag_subsets(env, flags):
     run(env, 57, D_RAGGED, 5, 250, seed=12, flags=flags, workers=[3, 56])
 
 
-@pytest.mark.parametrize("d", [147 * 4096, 147 * 4096 + 1, 148 * 4096 - 1])
+@pytest.mark.parametrize("d", [98 * 6144, 98 * 6144 + 1, 99 * 6144 - 1])
 def test_tile_boundaries(env, d):
     run(env, 60, d, 5, 250, seed=13, workers=[0, 59])
 
@@ -129,8 +128,9 @@ def test_heavy_tails(env):
     run(env, 57, D_RAGGED, 5, 250, seed=19, sigma=3.0, workers=[1])
 
 
-def test_unaligned_inputs_use_another_kernel(env):
-    run(env, 57, D_RAGGED, 5, 250, seed=20, misalign=1, workers=[0, 56], expect=None)
+def test_unaligned_inputs(env):
+    """Rows that start at an odd element (4-byte aligned only) take the same kernel: it loads 32 bits at a time."""
+    run(env, 57, D_RAGGED, 5, 250, seed=20, misalign=1, workers=[0, 56])
 
 
 def test_repeat_runs_agree(env):
@@ -141,7 +141,9 @@ def test_repeat_runs_agree(env):
 
 
 def test_last_kernel_names_follow_the_dispatch(env):
-    """Small jobs and jobs without a sketch are served by the other kernels, and the library says so."""
+    """Sketch requests are served by the list kernel whatever the size and alignment of the job;
+    requests without a sketch by the streaming kernel; sketches whose lists would be too short for
+    the schedule by the plain-load kernels - and the library says which one ran."""
     torch, oracle, F = env
     rng = np.random.default_rng(22)
     d, K, l, m = 50_000, 4, 5, 250
@@ -152,9 +154,14 @@ def test_last_kernel_names_follow_the_dispatch(env):
         w0 = torch.randn(d, device="cuda")
         st = torch.empty((K, ctx.state_len), device="cuda")
         ctx.fda_local_state(w, w0, None, 1 | 4, st)
-        assert ctx.fda_debug_last_kernel() == "k_local_state_staged"
+        assert ctx.fda_debug_last_kernel() == GATHER
         ctx.fda_local_state(w, w0, None, 1, st)
         assert ctx.fda_debug_last_kernel() == "k_local_state_linear"
         ctx.fda_local_state(w[:, 1:], w0[1:], None, 1 | 4, st)          # rows start at an odd element
-        assert ctx.fda_debug_last_kernel() == "k_local_state"
+        assert ctx.fda_debug_last_kernel() == GATHER
+        torch.cuda.synchronize()
+    with F.FdaContext(8, 2000, rand_coeffs(rng, 8), d_max=d, K_max=K) as ctx:   # no schedule for this sketch
+        st = torch.empty((K, ctx.state_len), device="cuda")
+        ctx.fda_local_state(w, w0, None, 1 | 4, st)
+        assert ctx.fda_debug_last_kernel() in ("k_local_state", "k_local_state_fast")
         torch.cuda.synchronize()
