@@ -15,7 +15,7 @@
  *   - plain C ABI; every function returns an fda_status and never throws or aborts;
  *   - unless a parameter says "host", pointers are DEVICE pointers to memory owned by the
  *     caller; the library never frees or reallocates caller memory;
- *   - the context owns its own device scratch (hash table, per-block partial sums);
+ *   - the context owns its own device scratch (list schedule, per-block partial sums);
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); calls
  *     enqueue work and return, unless stated otherwise;
  *   - arguments are validated on the host before anything is launched; an invalid call
@@ -82,14 +82,44 @@ typedef struct {
  *                  sign_i(j)   = +1 if ((((c3*j + c2)*j + c1)*j + c0) mod p) is even, else -1
  *                May be NULL when l == 0 (a context without sketch: state_len = 2).
  *   d_max, K_max largest model dimension / worker count later calls will use; they size
- *                the context's scratch (2*l bytes of hash table per index, plus partial
- *                sums).  Blocking: allocates, fills the hash table, synchronises.
+ *                the context's scratch.
+ * Device memory the context takes (fda_context_info reports the figures):
+ *   - per-block partial sums: (SM count) * l*m * 128 bytes plus 64 * (SM count) * max(K_max, 32) bytes;
+ *   - the list schedule of the sketch kernel, when the sketch allows one (tiles of at least 6*m
+ *     indices fit the shared memory): about 2.4 * l bytes per index of d_max (2.4 GB for
+ *     d_max = 2 * 10^8 and l = 5), built here in about 4 ms per million indices; it is dropped,
+ *     and sketch requests are then served by the slower plain-load kernels, when it would take
+ *     more than a third of the free device memory (see fda_create_limited for another cap);
+ *   - lazily, by the first call that needs them: a 16-bit hash table of 2*l bytes per index
+ *     (sketch requests without a schedule, fda_mean_state), d_max floats (fda_mean_state),
+ *     K_max*d_max floats of staging (fda_round_host).
+ * Blocking: allocates, builds the schedule, synchronises the device.
  * Errors: INVALID_ARG (out == NULL, l < 0 or > FDA_MAX_ROWS, m < 1 or > 32768 with l > 0,
  * d_max < 1 or >= 2^31, K_max < 1, coefficient out of range), UNSUPPORTED (l*m too large
  * for the shared-memory bins), NOMEM, CUDA.
  */
 fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
                       int64_t d_max, int K_max);
+
+/*
+ * fda_create with a cap on the list schedule (the paper has no counterpart): the schedule is
+ * kept only if it takes at most `schedule_limit_bytes` (and a third of the free device memory);
+ * 0 means no cap of the caller's (fda_create), a negative value builds no schedule at all.
+ * Other arguments and errors as fda_create.
+ */
+fda_status fda_create_limited(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
+                              int64_t d_max, int K_max, int64_t schedule_limit_bytes);
+
+/*
+ * What the context holds (the paper has no counterpart).  info (host, 8 values):
+ *   [0] device bytes the context owns now   [1] of which: the list schedule (0: none)
+ *   [2] 1 when sketch requests run on the list kernel, 0 when on the plain-load kernels
+ *   [3] indices per tile of the schedule    [4] bytes of a schedule that was built and dropped
+ *       for lack of memory (0: none)        [5] bytes of the lazily built 16-bit hash table
+ *   [6] microseconds fda_create spent on the schedule   [7] other lazily allocated bytes.
+ * Errors: INVALID_ARG (NULL).
+ */
+fda_status fda_context_info(const fda_ctx *ctx, int64_t *info);
 
 /* Free the context and its scratch.  Blocking (synchronises the device). NULL is a no-op. */
 fda_status fda_destroy(fda_ctx *ctx);
@@ -242,12 +272,11 @@ fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_hos
 
 /*
  * Name of the kernel that served the context's last fda_local_state call (the paper has no
- * counterpart): "k_local_state_gather" (sketch pass over per-cell index lists; 16-byte aligned inputs,
- * jobs of at least eight tiles per block whose lists average eight entries or more),
- * "k_local_state_staged" (compare-and-swap sketch pass on TMA-staged tiles; 16-byte aligned
- * inputs), "k_local_state_linear" (no sketch requested), "k_local_state" (everything else), or
- * "" before the first call.  The string is static; ctx == NULL gives "".  Tests and the
- * benchmark use it to say which kernel a number belongs to.
+ * counterpart): "k_local_state_gather" (sketch pass over per-cell index lists: every sketch request
+ * on a context that holds a list schedule), "k_local_state_linear" (no sketch requested),
+ * "k_local_state_fast" / "k_local_state" (sketch requests without a schedule: aligned rows with 5
+ * or 7 sketch rows / everything else), or "" before the first call.  The string is static;
+ * ctx == NULL gives "".  Tests and the benchmark use it to say which kernel a number belongs to.
  */
 const char *fda_debug_last_kernel(const fda_ctx *ctx);
 

@@ -20,7 +20,7 @@ FDA_MAX_ROWS = 16
 _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "FDA_ERR_CUDA",
            4: "FDA_ERR_NOMEM"}
 
-EXPORTS = ("fda_create", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
+EXPORTS = ("fda_create", "fda_create_limited", "fda_context_info", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
            "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel", "fda_debug_schedule",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
@@ -63,6 +63,10 @@ def load_library():
     lib = ctypes.CDLL(path)
     vp, i64, c_int, u32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint32, ctypes.c_float
     lib.fda_create.argtypes = [ctypes.POINTER(vp), c_int, c_int, c_int, vp, i64, c_int]
+    lib.fda_create_limited.argtypes = [ctypes.POINTER(vp), c_int, c_int, c_int, vp, i64, c_int, i64]
+    lib.fda_create_limited.restype = c_int
+    lib.fda_context_info.argtypes = [vp, vp]
+    lib.fda_context_info.restype = c_int
     lib.fda_destroy.argtypes = [vp]
     lib.fda_state_len.argtypes = [vp]
     lib.fda_state_len.restype = ctypes.c_size_t
@@ -144,7 +148,9 @@ def fda_local_state_linear_noalloc(w, w_t0, xi, flags: int, states, stream=None)
 class FdaContext:
     """Owner of an ``fda_ctx``.  Methods mirror the C entry points one to one."""
 
-    def __init__(self, l: int, m: int, hash_coeffs, d_max: int, K_max: int, device: int = 0):
+    def __init__(self, l: int, m: int, hash_coeffs, d_max: int, K_max: int, device: int = 0,
+                 schedule_limit_bytes: int | None = None):
+        """``schedule_limit_bytes``: None calls ``fda_create``; a number calls ``fda_create_limited``."""
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         coeffs = None
@@ -154,7 +160,11 @@ class FdaContext:
                 raise ValueError("hash_coeffs must hold 6*l values")
         self._coeffs = coeffs
         ptr = coeffs.ctypes.data_as(ctypes.c_void_p) if coeffs is not None else None
-        st = self._lib.fda_create(ctypes.byref(self._h), device, l, m, ptr, d_max, K_max)
+        if schedule_limit_bytes is None:
+            st = self._lib.fda_create(ctypes.byref(self._h), device, l, m, ptr, d_max, K_max)
+        else:
+            st = self._lib.fda_create_limited(ctypes.byref(self._h), device, l, m, ptr, d_max, K_max,
+                                              int(schedule_limit_bytes))
         if st != 0:
             self._h = ctypes.c_void_p()
             raise FdaError(st, "fda_create")
@@ -171,6 +181,14 @@ class FdaContext:
 
     def fda_last_error(self) -> str:
         return self._lib.fda_last_error(self._h).decode()
+
+    def fda_context_info(self) -> dict:
+        """What the context holds: see ``fda_context_info`` in include/fda.h."""
+        info = (ctypes.c_int64 * 8)()
+        self._check(self._lib.fda_context_info(self._h, info), "fda_context_info")
+        keys = ("device_bytes", "schedule_bytes", "list_kernel", "tile_indices", "schedule_dropped_bytes",
+                "table_bytes", "schedule_build_us", "other_lazy_bytes")
+        return dict(zip(keys, (int(v) for v in info)))
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h.value:

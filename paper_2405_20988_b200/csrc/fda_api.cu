@@ -1,4 +1,5 @@
 // C ABI of libfda: context management, argument validation, stream plumbing.
+#include <chrono>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -43,12 +44,10 @@ void free_device(fda_ctx *ctx)
 {
     cudaFree(ctx->coeffs_dev);
     cudaFree(ctx->tab);
-    cudaFree(ctx->tab32);
     cudaFree(ctx->sched);
     cudaFree(ctx->sched_off);
     cudaFree(ctx->part_sk);
     cudaFree(ctx->part_np);
-    cudaFree(ctx->err_flag);
     cudaFree(ctx->combine_scratch);
     cudaFree(ctx->combine_ticket);
     cudaFree(ctx->mean_model);
@@ -67,6 +66,12 @@ extern "C" {
 
 fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
                       int64_t d_max, int K_max)
+{
+    return fda_create_limited(out, device, l, m, hash_coeffs, d_max, K_max, 0);
+}
+
+fda_status fda_create_limited(fda_ctx **out, int device, int l, int m, const uint64_t *hash_coeffs,
+                              int64_t d_max, int K_max, int64_t schedule_limit_bytes)
 {
     if (!out) return FDA_ERR_INVALID_ARG;
     *out = nullptr;
@@ -103,37 +108,27 @@ fda_status fda_create(fda_ctx **out, int device, int l, int m, const uint64_t *h
     if (l > 0 && ctx->columns < 1) { delete ctx; return FDA_ERR_UNSUPPORTED; }
 
     ctx->max_blocks = ctx->n_sm * 4;
-    // padded by more than the widest tile of the staged kernel, so that a tile that starts below
+    ctx->sched_limit_bytes = schedule_limit_bytes;
+    // padded by more than the widest tile of the plain-load kernels, so that a tile that starts below
     // d_max never reads past the table (entries past d_max are valid hashes of those indices)
     ctx->tab_stride = (d_max + 1024 + 63) / 64 * 64;
     ctx->part_sk_floats = l > 0 ? (size_t)ctx->n_sm * ctx->lm * 32 : 0;
     if (l > 0) {
         e = cudaMalloc(&ctx->coeffs_dev, sizeof(uint64_t) * 6 * l);
-        if (e == cudaSuccess) e = cudaMalloc(&ctx->tab, sizeof(uint16_t) * (size_t)l * ctx->tab_stride);
         if (e == cudaSuccess)
             e = cudaMemcpy(ctx->coeffs_dev, ctx->coeffs_host, sizeof(uint64_t) * 6 * l, cudaMemcpyHostToDevice);
-        // the list schedule first: where it exists the staged kernel only serves jobs of fewer than
-        // eight tiles per block, and its table need not cover more indices than those
-        if (e == cudaSuccess) e = fda_build_list_schedule(ctx, nullptr);
-        ctx->tab32_stride = ctx->tab_stride;
-        if (ctx->sched) {
-            const int64_t cap = ((int64_t)8 * ctx->n_sm * ctx->sched_T + 1024 + 63) / 64 * 64;
-            if (cap < ctx->tab32_stride) ctx->tab32_stride = cap;
+        if (e == cudaSuccess && schedule_limit_bytes >= 0) {
+            const auto t0 = std::chrono::steady_clock::now();
+            e = fda_build_list_schedule(ctx, nullptr);
+            ctx->sched_build_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
         }
-        // the 32-bit table serves the staged sketch kernel only, which needs all l*m bins with 32
-        // columns plus its ring in shared memory
-        if (e == cudaSuccess && (size_t)ctx->lm * 128 + 16384 <= (size_t)ctx->smem_optin)
-            e = cudaMalloc(&ctx->tab32, sizeof(uint32_t) * (size_t)l * ctx->tab32_stride);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
     }
     ctx->part_np_doubles = (size_t)ctx->max_blocks * (size_t)(K_max > 32 ? K_max : 32) * 2;
     if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * ctx->part_np_doubles);
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->err_flag, sizeof(unsigned int));
-    if (e == cudaSuccess) e = cudaMemset(ctx->err_flag, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_scratch, sizeof(double) * (2 + FDA_MAX_ROWS));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->combine_ticket, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(ctx->combine_ticket, 0, sizeof(unsigned int));
-    if (e == cudaSuccess) e = fda_launch_build_table(ctx, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         const fda_status st = e == cudaErrorMemoryAllocation ? FDA_ERR_NOMEM : FDA_ERR_CUDA;
@@ -222,14 +217,8 @@ fda_status fda_combine_estimate(fda_ctx *ctx, const float *states, int K, int va
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = fda_launch_combine(ctx, states, K, variant, epsilon, theta, est_dev, s);
     if (e == cudaSuccess && est_host) {
-        unsigned int flag = 0;
         e = cudaMemcpyAsync(est_host, est_dev, sizeof(fda_estimate), cudaMemcpyDeviceToHost, s);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(&flag, ctx->err_flag, sizeof(flag), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-        if (e == cudaSuccess && flag != 0) {
-            cudaMemsetAsync(ctx->err_flag, 0, sizeof(flag), s);
-            return fail(ctx, FDA_ERR_CUDA, "a device-side wait of an earlier fda_local_state ran out; its states are invalid");
-        }
     }
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fda_combine_estimate");
     return FDA_OK;
@@ -377,6 +366,30 @@ fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_hos
     const size_t n = capacity < (size_t)info[3] ? capacity : (size_t)info[3];
     e = cudaMemcpy(record_host, ctx->sched + off[0], n, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }
+    return FDA_OK;
+}
+
+fda_status fda_context_info(const fda_ctx *ctx, int64_t *info)
+{
+    if (!ctx || !info) return FDA_ERR_INVALID_ARG;
+    const int64_t table = ctx->tab ? (int64_t)(sizeof(uint16_t) * (size_t)ctx->l * ctx->tab_stride) : 0;
+    const int64_t sched = ctx->sched ? (int64_t)(ctx->sched_bytes + sizeof(uint64_t) * (size_t)(ctx->sched_tiles + 1)) : 0;
+    const int64_t partial = (int64_t)(sizeof(float) * ctx->part_sk_floats + sizeof(double) * ctx->part_np_doubles +
+                                      sizeof(double) * (2 + FDA_MAX_ROWS) + sizeof(unsigned int)) +
+                            (ctx->coeffs_dev ? (int64_t)sizeof(uint64_t) * 6 * ctx->l : 0);
+    const int64_t mean = ctx->mean_model ? (int64_t)sizeof(float) * ((ctx->d_max + 3) / 4 * 4) : 0;
+    int64_t stage = 0;
+    if (ctx->stage_w)
+        stage = (int64_t)sizeof(float) * ((int64_t)ctx->K_max * ctx->stage_stride + 2 * ctx->stage_stride +
+                                          (int64_t)ctx->K_max * (2 + ctx->lm)) + (int64_t)sizeof(fda_estimate);
+    info[0] = table + sched + partial + mean + stage;
+    info[1] = sched;
+    info[2] = ctx->sched ? 1 : 0;
+    info[3] = ctx->sched_T;
+    info[4] = (int64_t)ctx->sched_skipped_bytes;
+    info[5] = table;
+    info[6] = (int64_t)(ctx->sched_build_ms * 1000.0);
+    info[7] = mean + stage;
     return FDA_OK;
 }
 

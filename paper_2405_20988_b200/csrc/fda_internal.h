@@ -22,6 +22,7 @@ constexpr int kListPadRows = 8;        // zero rows behind the tile, one per ban
 constexpr int kListBatch = 1024;       // indices a producer step covers; tiles are multiples of it
 constexpr int kListMaxTile = 7168;     // rows + pad rows must fit 13 bits
 constexpr int kListMinTilesPerBlock = 1;
+constexpr int kListSmemHead = 1088;    // counters and the producer warps' fp64 sums in front of the item tables
 
 // byte offsets inside the schedule record of a tile with `items` items
 inline __host__ __device__ size_t fda_sched_cells_off(uint32_t items) { return ((size_t)16 + 8 * (size_t)items + 63) / 64 * 64; }
@@ -34,7 +35,7 @@ inline __host__ __device__ uint32_t fda_list_row(uint32_t r) { return r ^ ((r >>
 inline int fda_list_table_bytes(int ni_max) { return (16 + 8 * ni_max + 15) / 16 * 16; }
 inline size_t fda_list_smem_bytes(int l, int m, int T, int ni_max)
 {
-    return 576 + 2 * (size_t)fda_list_table_bytes(ni_max) + (size_t)l * m * kListWorkers * 4 +
+    return kListSmemHead + 2 * (size_t)fda_list_table_bytes(ni_max) + (size_t)l * m * kListWorkers * 4 +
            2 * (size_t)(T + kListPadRows) * kListWorkers * 4;
 }
 
@@ -49,10 +50,8 @@ struct fda_ctx {
     int columns = 0;           // lane-private columns per cell in the shared-memory bins
     // device scratch
     uint64_t *coeffs_dev = nullptr;   // 6*l
-    uint16_t *tab = nullptr;          // l planes of tab_stride entries
-    uint32_t *tab32 = nullptr;        // same hash as cell index | sign<<31 (staged sketch kernel)
+    uint16_t *tab = nullptr;          // l planes of tab_stride entries; built by the first call that needs it
     int64_t tab_stride = 0;
-    int64_t tab32_stride = 0;         // entries per plane of tab32: the indices the staged kernel may be asked for
     float *part_sk = nullptr;         // per-block sketch partials
     size_t part_sk_floats = 0;
     double *part_np = nullptr;        // per-block (norm, projection) partials
@@ -69,15 +68,6 @@ struct fda_ctx {
     int64_t sched_tiles = 0;
     double sched_build_ms = 0.0;      // host time spent building it
     float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
-    // tensor maps of the last staged launch (encoding four maps costs several microseconds of
-    // host time, which matters for small models); valid while the key below matches
-    alignas(64) unsigned char tmap_cache[4][128] = {};
-    struct {
-        const void *w = nullptr, *w_t0 = nullptr, *xi = nullptr;
-        int64_t row_stride = 0, d = 0;
-        int K = 0, bx = 0, Kg = 0;
-    } tmap_key;
-    unsigned int *err_flag = nullptr;  // set by a kernel whose bounded wait ran out
     double *combine_scratch = nullptr;        // 2 + FDA_MAX_ROWS doubles: S-bar[0..1] and the row norms
     unsigned int *combine_ticket = nullptr;   // blocks of the combine kernel that have finished (0 between launches)
     // staging for fda_round_host (lazy)
@@ -90,7 +80,7 @@ struct fda_ctx {
 };
 
 // ---- launchers (each returns the cudaError_t of its launches) -------------------------
-cudaError_t fda_launch_build_table(const fda_ctx *ctx, cudaStream_t s);
+cudaError_t fda_ensure_table(fda_ctx *ctx, cudaStream_t s);   // allocates and fills ctx->tab on first use
 cudaError_t fda_launch_read_probe(const fda_ctx *ctx, const float *src, int64_t n, float *sum_out,
                                   cudaStream_t s);
 cudaError_t fda_launch_debug_hash(const fda_ctx *ctx, int64_t j0, int64_t n, uint16_t *buckets,
@@ -98,9 +88,6 @@ cudaError_t fda_launch_debug_hash(const fda_ctx *ctx, int64_t j0, int64_t n, uin
 cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s);
-cudaError_t fda_launch_local_state_staged(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
-                                          int64_t d, const float *w_t0, const float *xi,
-                                          uint32_t flags, float *states, cudaStream_t s);
 cudaError_t fda_build_list_schedule(fda_ctx *ctx, cudaStream_t s);   // allocates and fills ctx->sched when it fits
 cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,

@@ -465,14 +465,16 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
                                    int64_t d, const float *w_t0, const float *xi, uint32_t flags,
                                    float *states, cudaStream_t s)
 {
-    {   // sketch requests: the list kernel when its schedule exists and the job is large enough, else
-        // the staged kernel (aligned inputs); requests without a sketch: the streaming kernel
+    {   // sketch requests: the list kernel when the context holds its schedule; requests without a
+        // sketch: the streaming kernel; everything else: the plain-load kernels below
         cudaError_t e = fda_launch_local_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
         if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_gather"; return e; }
-        e = fda_launch_local_state_staged(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_staged"; return e; }
         e = fda_launch_local_state_linear(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
         if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_linear"; return e; }
+    }
+    if (flags & FDA_STATE_SKETCH) {
+        const cudaError_t e = fda_ensure_table(ctx, s);
+        if (e != cudaSuccess) return e;
     }
     ctx->last_ls_kernel = "k_local_state";
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;

@@ -33,14 +33,18 @@
 namespace {
 
 constexpr int GW = kListWorkers;
-constexpr int kProducerWarps = 8;
-constexpr int kWalkerWarps = 20;
+#ifndef FDA_PW
+#define FDA_PW 8
+#define FDA_WW 20
+#define FDA_DEPTH 1
+#endif
+constexpr int kProducerWarps = FDA_PW;
+constexpr int kWalkerWarps = FDA_WW;
 constexpr int kThreads = (kProducerWarps + kWalkerWarps) * 32;
-constexpr int kDepth = 4;                      // batches a producer thread keeps in flight
-constexpr int kProducerRegs = 112, kWalkerRegs = 56;
-static_assert(kProducerRegs * kProducerWarps + kWalkerRegs * kWalkerWarps <= 72 * (kProducerWarps + kWalkerWarps), "register split exceeds the launch");
+constexpr int kDepth = FDA_DEPTH;                      // batches a producer thread keeps in flight
 constexpr int kChunksAhead = 8;                // entry chunks (four steps each) a walker loads before it walks them
-static_assert(kProducerWarps * 32 * 4 == kListBatch, "a batch is four consecutive indices per producer thread");
+constexpr int kBatch = kProducerWarps * 32 * 4;   // a batch is four consecutive indices per producer thread
+static_assert(kProducerWarps <= 16 && kListBatch % kBatch == 0, "tiles are whole batches; the fp64 sums have room for 16 producer warps");
 
 struct ListParams {
     const float *w, *w_t0, *xi;
@@ -96,6 +100,18 @@ __device__ __forceinline__ float4 load_quad(const float *ptr, bool vec, int n)
     v.x = load1(ptr, n > 0); v.y = load1(ptr + 1, n > 1); v.z = load1(ptr + 2, n > 2); v.w = load1(ptr + 3, n > 3);
     return v;
 }
+__device__ __forceinline__ uint4 load_u4(const void *ptr)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
+    return v;
+}
+__device__ __forceinline__ unsigned long long load_u64(const void *ptr)
+{
+    unsigned long long v;
+    asm volatile("ld.global.nc.u64 %0, [%1];" : "=l"(v) : "l"(ptr));
+    return v;
+}
 __device__ __forceinline__ void store_row(uint32_t addr, float x, float y, float z, float w)
 {
     asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
@@ -140,7 +156,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem_raw);
     int *ctr = reinterpret_cast<int *>(smem_raw);
     double *sums = reinterpret_cast<double *>(smem_raw + 64);
-    const uint32_t tab_off = 576;
+    const uint32_t tab_off = kListSmemHead;
     const uint32_t bins_off = tab_off + 2u * (uint32_t)p.tab_bytes;
     const uint32_t ut_off = bins_off + (uint32_t)lm * 16u;
     const uint32_t ut_bytes = (uint32_t)(T + kListPadRows) * 16u;
@@ -157,12 +173,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
 
     const int64_t n_tiles = p.tiles > c ? (p.tiles - c + p.cpg - 1) / p.cpg : 0;
 
-    // The block is launched with 72 registers per thread; the walkers give some back and the
-    // producers take them: their registers are the landing zone of the loads in flight
-    // (8 warps x 32 lanes x kDepth batches x 5 or 6 x 16 bytes), and what is in flight bounds
-    // the memory bandwidth.  112 * 256 + 56 * 640 = 72 * 896.
     if (warp < kProducerWarps) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kProducerRegs));
         // =============================== producers ===============================
         const int pt = tid;                                   // quad of indices inside a batch
         // rows of the group; workers past K alias the group's first row (their sums are computed
@@ -197,6 +208,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
         };
         prefetch_tile(0);
         prefetch_tile(1);
+        // head of the schedule record of the tile being stored (the walkers' item table) and the
+        // record offsets of the next tile, loaded one and two tiles ahead of their use
+        uint4 tabv = make_uint4(0u, 0u, 0u, 0u);
+        unsigned long long off0 = load_u64(p.sched_off + c), off1 = load_u64(p.sched_off + c + 1);
+        if (pt * 16 < p.tab_bytes) tabv = load_u4(p.sched + off0 + pt * 16);
+        if (n_tiles > 1) { off0 = load_u64(p.sched_off + c + p.cpg); off1 = load_u64(p.sched_off + c + p.cpg + 1); }
         auto issue = [&](int slot) {
             if (n_i < n_tiles) {
                 const float *q = wbase + j_i;
@@ -214,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
                     w0v[slot] = load_quad<false>(p.w_t0 + j_i, vec, n);
                     if (LINEAR) xv[slot] = load_quad<false>(p.xi + j_i, vec, n);
                 }
-                j_i += kListBatch;
+                j_i += kBatch;
                 if (++b_i == p.nb) { b_i = 0; ++n_i; j_i += wrap; end_i += wrap + T; }
             }
         };
@@ -223,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
             // rows 4*pt .. 4*pt+3 of the batch; row r is stored at r ^ ((r >> 3) & 3), so that the
             // eight lanes of a store pass hit eight different bank groups (the schedule's entries
             // hold the swizzled row)
-            const uint32_t r0 = (uint32_t)(b_c * kListBatch + 4 * pt);
+            const uint32_t r0 = (uint32_t)(b_c * kBatch + 4 * pt);
             const uint32_t dst0 = smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 16u;
             const uint32_t sw = (r0 >> 3) & 3u;
 #pragma unroll
@@ -259,18 +276,21 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
                     }
                     nf[k] = 0.f; pf[k] = 0.f;
                 }
-                const int64_t tile = c + n_c * p.cpg;
-                const unsigned char *rec = p.sched + p.sched_off[tile];
+                // the table of this tile (loaded a tile ago), the loads of the next one, the offsets
+                // of the one after: nothing here waits for memory
                 if (pt * 16 < p.tab_bytes)
-                    *reinterpret_cast<uint4 *>(smem_raw + tab_off + (size_t)buf * p.tab_bytes + pt * 16) =
-                        __ldg(reinterpret_cast<const uint4 *>(rec) + pt);
+                    *reinterpret_cast<uint4 *>(smem_raw + tab_off + (size_t)buf * p.tab_bytes + pt * 16) = tabv;
                 if (pt == 0) ctr[buf] = 0;
-                if (n_c + 1 < n_tiles) {                      // the next record into L2 ahead of its walk
-                    const int64_t nt = tile + p.cpg;
-                    const unsigned char *nrec = p.sched + p.sched_off[nt];
-                    const uint32_t nbytes = (uint32_t)(p.sched_off[nt + 1] - p.sched_off[nt]);
-                    for (uint32_t o = (uint32_t)pt * 128u; o < nbytes; o += 256u * 128u)
+                if (n_c + 1 < n_tiles) {
+                    const unsigned char *nrec = p.sched + off0;
+                    if (pt * 16 < p.tab_bytes) tabv = load_u4(nrec + pt * 16);
+                    for (uint64_t o = (uint64_t)pt * 128u; o < off1 - off0; o += (uint64_t)kProducerWarps * 32u * 128u)   // the record into L2 ahead of its walk
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(nrec + o));
+                }
+                if (n_c + 2 < n_tiles) {
+                    const int64_t t2 = c + (n_c + 2) * p.cpg;
+                    off0 = load_u64(p.sched_off + t2);
+                    off1 = load_u64(p.sched_off + t2 + 1);
                 }
                 prefetch_tile(n_c + 2);
                 block_barrier();
@@ -287,7 +307,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
             }
         }
     } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kWalkerRegs));
         // =============================== walkers ===============================
         for (int64_t n = 0; n < n_tiles; ++n) {
             block_barrier();                                   // tile n is stored, tile n - 1 is walked
@@ -424,7 +443,8 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     p.K = K; p.d = d; p.have_xi = xi_used != nullptr;
     p.vec = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) && (row_stride % 4 == 0);
     p.l = ctx->l; p.m = ctx->m;
-    p.T = ctx->sched_T; p.nb = p.T / kListBatch;
+    p.T = ctx->sched_T; p.nb = p.T / kBatch;
+    if (p.T % kBatch != 0) return cudaErrorNotSupported;
     p.sched = ctx->sched; p.sched_off = ctx->sched_off;
     p.part_sk = ctx->part_sk; p.part_np = ctx->part_np;
     p.tiles = (d + p.T - 1) / p.T;
@@ -441,7 +461,7 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
         (size_t)blocks * GW * 2 > ctx->part_np_doubles)
         return cudaErrorNotSupported;
     const size_t smem = fda_list_smem_bytes(p.l, p.m, p.T, ctx->sched_ni_max);
-    if (smem > (size_t)ctx->smem_optin || 256 * 16 < p.tab_bytes) return cudaErrorNotSupported;
+    if (smem > (size_t)ctx->smem_optin || kProducerWarps * 32 * 16 < p.tab_bytes) return cudaErrorNotSupported;
 
     auto kern = xi_used ? k_local_state_gather<true> : k_local_state_gather<false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin);

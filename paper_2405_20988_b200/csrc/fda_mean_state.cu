@@ -342,6 +342,10 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
 {
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
+    if (sketch) {                // first use: the 16-bit hash table
+        const cudaError_t e = fda_ensure_table(ctx, s);
+        if (e != cudaSuccess) return e;
+    }
     if (!ctx->mean_model) {      // first use: d_max floats of scratch for the average drift
         cudaError_t e = cudaMalloc(&ctx->mean_model, sizeof(float) * (size_t)((ctx->d_max + 3) / 4 * 4));
         if (e != cudaSuccess) return e;
