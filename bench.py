@@ -2,13 +2,15 @@
 """Benchmark of the FDA hot path on B200: one step = local states -> combine/estimate ->
 K-way model average (in-place sync) over one synthetic workload resident in HBM.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..7] [--impl reference]
 
 Prints ONE JSON line.  ``value`` is params*workers/s of the whole step (K*d elements per
 step / device time per step, CUDA events on the launching stream); ``roofline`` describes
 the dominant kernel (the fused local-state pass); ``e2e`` is the same metric through
 ``fda_round_host`` (pinned host buffers, copies inside the timed region); ``cpu_baseline``
-is the CPU oracle timed on a bounded sample of the same workload.
+is the CPU oracle timed on a bounded sample of the same workload; ``also`` (default workload
+only) holds the step, kernel times and roofline of the 20M-parameter workload, measured in the
+same process after the main one is freed.
 
 With ``--impl reference`` the CPU oracle itself is the timed arm (rank 0 only).
 Under torchrun every rank runs an independent replica of the workload on its own GPU (the
@@ -42,9 +44,36 @@ NOMINAL_HBM_GBS = 8000.0               # the data-sheet figure, quoted beside th
 SMEM_CAS_UPDATES_PER_CLK_SM = 6.8     # measured on B200: bare fp32 shared-memory atomicAdd loop, 1024 threads
 SMEM_GATHER_UPDATES_PER_CLK_SM = 32.0  # one 4-byte shared-memory read per update at 128 bytes per clock and SM
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_local_state launch from the ncu
-# capture summarised under profiles/ (None: not captured for the kernel as it stands).
-LOCAL_STATE_TRAFFIC_BYTES = {1: None, 2: None, 3: 949_400_000, 4: 5_165_200_000, 5: 9_579_100_000}
+# dram__bytes_read.sum + dram__bytes_write.sum of one sketch-pass launch come from the ncu launch
+# lists summarised under profiles/: profiles/traffic.json names, per workload, the bytes, the
+# summary file and the sha256 of the kernel sources the capture was taken with.  When the sources
+# have changed since, the figure is stale and the bench line says null.
+KERNEL_SOURCES = ("paper_2405_20988_b200/csrc/fda_local_state_gather.cu", "paper_2405_20988_b200/csrc/fda_sched.cu",
+                  "paper_2405_20988_b200/csrc/fda_internal.h")
+
+
+def kernel_sources_sha256() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_traffic(workload: int):
+    """(bytes per launch or None, where the figure comes from)"""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            tab = json.load(f)
+        ent = tab["workloads"].get(str(workload))
+        if ent is None:
+            return None, "no capture for this workload"
+        if tab["sources_sha256"] != kernel_sources_sha256():
+            return None, "kernel sources changed since %s was captured" % ent["profile"]
+        return ent["bytes"], ent["profile"]
+    except (OSError, KeyError, ValueError):
+        return None, "profiles/traffic.json missing"
 
 
 def secondary_roofline(kernel, updates_per_s, n_sm, sm_mhz):
@@ -181,86 +210,123 @@ def run_ours(args, rank, world, local_rank):
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = S.WORKLOADS[args.workload]
-    d, K = wl.d, wl.K
     cores = host_cores()
     gen_threads = max(1, cores // max(1, world))
-    w_t0_np = S.last_global_model(wl)
-    xi_np = S.unit_direction(wl)
-    coeffs = S.hash_coefficients(wl.seed, wl.l)
-    stride = S.row_stride(d)
-    w_pin = torch.empty((K, stride), dtype=torch.float32).pin_memory()
-    S.worker_models(wl, w_t0_np, out=w_pin.numpy(), threads=gen_threads)
-    w0_pin = torch.from_numpy(w_t0_np).pin_memory()
-    xi_pin = torch.from_numpy(xi_np).pin_memory()
 
-    ctx = F.FdaContext(wl.l, wl.m, coeffs, d_max=d, K_max=K, device=local_rank)
-    w_src = w_pin.to(dev, non_blocking=True)          # pristine copies (restored before each step)
-    w0_src = w0_pin.to(dev, non_blocking=True)
-    xi = xi_pin.to(dev, non_blocking=True)
-    w = torch.empty_like(w_src)
-    w0 = torch.empty_like(w0_src)
-    states = torch.empty((K, ctx.state_len), dtype=torch.float32, device=dev)
-    est_buf = ctx.new_estimate_buffer(dev)
-    theta, eps = float(wl.thetas[-1]), float(np.float32(wl.epsilon))
-    stream = torch.cuda.current_stream()
+    class Run:
+        """One workload resident in HBM with its context, and the timed steps on it."""
 
-    ls_kernel = [""]       # the kernel the library picked for the sketch pass (asked after each launch)
+    def setup_and_time(workload, steps, warmup):
+        r = Run()
+        wl = S.WORKLOADS[workload]
+        d, K = wl.d, wl.K
+        r.wl, r.d, r.K = wl, d, K
+        r.w_t0_np = S.last_global_model(wl)
+        r.xi_np = S.unit_direction(wl)
+        r.coeffs = S.hash_coefficients(wl.seed, wl.l)
+        stride = S.row_stride(d)
+        r.stride = stride
+        r.w_pin = torch.empty((K, stride), dtype=torch.float32).pin_memory()
+        S.worker_models(wl, r.w_t0_np, out=r.w_pin.numpy(), threads=gen_threads)
+        r.w0_pin = torch.from_numpy(r.w_t0_np).pin_memory()
+        xi_pin = torch.from_numpy(r.xi_np).pin_memory()
 
-    def step(timed):
-        # the sync of the previous step made all models equal: put the drifted models back
-        w.copy_(w_src)
-        w0.copy_(w0_src)
-        return step_events()
-
-    def step_events():
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-        ev[0].record(stream)
-        ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
-        ls_kernel[0] = ctx.fda_debug_last_kernel()
-        ev[1].record(stream)
-        ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, eps, theta, est_buf, want_host=False)
-        ev[2].record(stream)
-        ctx.fda_average_models(w[:, :d], w0, est_buf, F.FDA_AVG_BROADCAST)
-        ev[3].record(stream)
-        return ev
-
-    def timed_run():
-        sampler = ClockSampler(local_rank)      # spans warm-up and timed steps (all under load)
-        sampler.start()
-        for _ in range(args.warmup):
-            step(False)
         torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
-        evs = [step(True) for _ in range(args.steps)]
-        torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
-        late = False
-        if not sampler.lines:
-            # the timed region was shorter than one sampling period: keep the same load running
-            # (untimed) until the sampler has seen it
-            late = True
-            t_end = time.perf_counter() + 1.5
-            while len(sampler.lines) < 2 and time.perf_counter() < t_end:
-                for _ in range(20):
-                    step(False)
-                torch.cuda.synchronize()
-        clocks = sampler.stop()
-        if late:
-            clocks["sampled"] = "under the same load right after the timed steps (they took less than one sample period)"
-        parts = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in evs])
-        return parts, clocks
+        t0 = time.perf_counter()
+        ctx = F.FdaContext(wl.l, wl.m, r.coeffs, d_max=d, K_max=K, device=local_rank)
+        r.create_ms = (time.perf_counter() - t0) * 1e3
+        r.ctx = ctx
+        r.w_src = r.w_pin.to(dev, non_blocking=True)          # pristine copies (restored before each step)
+        r.w0_src = r.w0_pin.to(dev, non_blocking=True)
+        r.xi = xi_pin.to(dev, non_blocking=True)
+        r.w = torch.empty_like(r.w_src)
+        r.w0 = torch.empty_like(r.w0_src)
+        r.states = torch.empty((K, ctx.state_len), dtype=torch.float32, device=dev)
+        r.est_buf = ctx.new_estimate_buffer(dev)
+        r.theta, r.eps = float(wl.thetas[-1]), float(np.float32(wl.epsilon))
+        r.ls_kernel = ""       # the kernel the library picked for the sketch pass (asked after each launch)
+        w, w0, states, est_buf = r.w, r.w0, r.states, r.est_buf
 
-    parts, clocks = timed_run()
-    if clocks_rejected(clocks):
+        def step_events():
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record(stream)
+            ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
+            r.ls_kernel = ctx.fda_debug_last_kernel()
+            ev[1].record(stream)
+            ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, r.eps, r.theta, est_buf, want_host=False)
+            ev[2].record(stream)
+            ctx.fda_average_models(w[:, :d], w0, est_buf, F.FDA_AVG_BROADCAST)
+            ev[3].record(stream)
+            return ev
+
+        def step(timed):
+            # the sync of the previous step made all models equal: put the drifted models back
+            w.copy_(r.w_src)
+            w0.copy_(r.w0_src)
+            return step_events()
+
+        r.step, r.step_events = step, step_events
+
+        def timed_run():
+            sampler = ClockSampler(local_rank)      # spans warm-up and timed steps (all under load)
+            sampler.start()
+            for _ in range(warmup):
+                step(False)
+            torch.cuda.synchronize()
+            if dist:
+                dist.barrier()
+            torch.cuda.synchronize()
+            evs = [step(True) for _ in range(steps)]
+            torch.cuda.synchronize()
+            if dist:
+                dist.barrier()
+            late = False
+            if not sampler.lines:
+                # the timed region was shorter than one sampling period: keep the same load running
+                # (untimed) until the sampler has seen it
+                late = True
+                t_end = time.perf_counter() + 1.5
+                while len(sampler.lines) < 2 and time.perf_counter() < t_end:
+                    for _ in range(20):
+                        step(False)
+                    torch.cuda.synchronize()
+            clocks = sampler.stop()
+            if late:
+                clocks["sampled"] = "under the same load right after the timed steps (they took less than one sample period)"
+            parts = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in evs])
+            return parts, clocks
+
         parts, clocks = timed_run()
-        clocks["remeasured"] = True
-    est = F.Estimate.from_buffer_copy(bytes(est_buf.cpu().numpy()))
-    if not est.trigger:
-        raise SystemExit("bench: the round did not trigger; the average was not timed")
+        if clocks_rejected(clocks):
+            parts, clocks = timed_run()
+            clocks["remeasured"] = True
+        r.parts, r.clocks = parts, clocks
+        r.est = F.Estimate.from_buffer_copy(bytes(est_buf.cpu().numpy()))
+        if not r.est.trigger:
+            raise SystemExit("bench: the round did not trigger; the average was not timed")
+        r.info = ctx.fda_context_info()
+        return r
+
+    def roofline_of(r, peak, peak_kind):
+        """The sketch pass of a run against the HBM roofline (algorithmic bytes: w, w_t0 read; states written)."""
+        ls_ms = float(r.parts[:, 0].mean())
+        algo_bytes = 4.0 * (r.K * r.d + r.d + r.K * r.ctx.state_len)
+        achieved = algo_bytes / (ls_ms * 1e-3) / 1e9
+        traffic, traffic_src = measured_traffic(r.wl_id)
+        return {"kernel": r.ls_kernel, "bound": "hbm", "achieved": achieved, "peak": peak,
+                "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                "algorithmic_bytes": algo_bytes, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                "traffic": traffic, "traffic_source": traffic_src}
+
+    stream = torch.cuda.current_stream()
+    run = setup_and_time(args.workload, args.steps, args.warmup)
+    run.wl_id = args.workload
+    wl, d, K, ctx = run.wl, run.d, run.K, run.ctx
+    w, w0, w_src, w0_src, xi, states, est_buf = run.w, run.w0, run.w_src, run.w0_src, run.xi, run.states, run.est_buf
+    w_pin, w0_pin, w_t0_np, xi_np, coeffs, stride = run.w_pin, run.w0_pin, run.w_t0_np, run.xi_np, run.coeffs, run.stride
+    theta, eps, parts, clocks, est = run.theta, run.eps, run.parts, run.clocks, run.est
+    ls_kernel = [run.ls_kernel]
+    step_events = run.step_events
 
     # ---- the LinearFDA flavour of the local-state pass, timed beside the headline step ----
     w.copy_(w_src)
@@ -394,11 +460,7 @@ def run_ours(args, rank, world, local_rank):
                            "frac_of_peak": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9 / peak,
                            "H": mean_est["H"], "note": "fda_mean_state: S-bar in one pass, no per-worker sketches"},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
-            "roofline": {"kernel": ls_kernel[0], "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
-                         "algorithmic_bytes": algo_bytes,
-                         "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
-                         "traffic": LOCAL_STATE_TRAFFIC_BYTES.get(args.workload)},
+            "roofline": roofline_of(run, peak, peak_kind),
             # what binds the sketch pass next to HBM: the shared-memory traffic of the l updates per
             # element (gather kernel: one 4-byte read each, 32 per clock and SM at best; the
             # compare-and-swap kernels: a measured 6.8 adds per clock and SM)
@@ -410,8 +472,42 @@ def run_ours(args, rank, world, local_rank):
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "api": "fda_round_host"},
             "gpu_launches": 4 * args.steps,
             "clocks": clocks,
+            "context": {"device_bytes": run.info["device_bytes"], "schedule_bytes": run.info["schedule_bytes"],
+                        "tile_indices": run.info["tile_indices"], "table_bytes": run.info["table_bytes"],
+                        "schedule_dropped_bytes": run.info["schedule_dropped_bytes"],
+                        "fda_create_ms": run.create_ms, "schedule_build_ms": run.info["schedule_build_us"] / 1e3,
+                        "note": "as reported by fda_context_info after the timed steps (before the lazily "
+                                "allocated scratch of fda_mean_state and fda_round_host)"},
+            "also": None,
         }
     ctx.close()
+    # ---- the other roofline workload named by the target (20M parameters, K = 60, sketch 7 x 500),
+    # measured in the same process once the main workload is freed ----
+    if rank == 0 and world == 1 and args.workload == 5 and not args.skip_also:
+        del run, w, w0, w_src, w0_src, xi, states, est_buf, w_pin, w0_pin, st_pin, mean_state
+        torch.cuda.empty_cache()
+        r4 = setup_and_time(4, max(3, min(args.steps, 20)), 3)
+        r4.wl_id = 4
+        p4 = r4.parts.mean(axis=0)
+        out["also"] = {
+            "config": {"workload": "4:%s d=%d K=%d sketch=%dx%d eps=%.4f theta=%g" %
+                                   (r4.wl.name, r4.d, r4.K, r4.wl.l, r4.wl.m, r4.wl.epsilon, r4.theta)},
+            "steps": int(r4.parts.shape[0]), "warmup": 3,
+            "ms_per_step": float(r4.parts.sum(axis=1).mean()),
+            "value": r4.K * r4.d / (float(r4.parts.sum(axis=1).mean()) * 1e-3), "unit": UNIT,
+            "kernels_ms": {"local_state": float(p4[0]), "combine": float(p4[1]), "average": float(p4[2])},
+            "roofline": roofline_of(r4, peak, peak_kind),
+            "average_only": {"gbs": 4.0 * (2 * r4.K * r4.d + r4.d) / (float(p4[2]) * 1e-3) / 1e9,
+                             "frac_of_peak": 4.0 * (2 * r4.K * r4.d + r4.d) / (float(p4[2]) * 1e-3) / 1e9 / peak},
+            "secondary_roofline": secondary_roofline(r4.ls_kernel, r4.K * r4.d * r4.wl.l / (float(p4[0]) * 1e-3), n_sm,
+                                                     r4.clocks.get("sm_mhz") or 1965.0),
+            "estimate": {"H": r4.est.H, "trigger": int(r4.est.trigger)},
+            "context": {"device_bytes": r4.info["device_bytes"], "schedule_bytes": r4.info["schedule_bytes"],
+                        "tile_indices": r4.info["tile_indices"], "fda_create_ms": r4.create_ms},
+            "clocks": r4.clocks,
+        }
+        out["gpu_launches"] += 4 * int(r4.parts.shape[0])
+        r4.ctx.close()
     if dist:
         dist.barrier()
         dist.destroy_process_group()
@@ -459,6 +555,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer leg (profiling runs)")
+    ap.add_argument("--skip-also", action="store_true", help="omit the second roofline workload (profiling runs)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
