@@ -301,7 +301,10 @@ const char *fda_debug_last_kernel(const fda_ctx *ctx);
  * launched.  Neither this call nor anything it uses calls cudaMalloc, cudaFree or an
  * allocating library routine.  The first call on a device looks up the device address of the
  * scratch array (cudaGetSymbolAddress); make that first call before starting any stream
- * capture.  All calls on a device share the one scratch array: two calls whose kernels
+ * capture, and make it at start-up: with CUDA's lazy module loading the library's kernels and
+ * the scratch array itself are placed in device memory when they are first touched, i.e. by
+ * that first call, which therefore still needs a little free device memory - later calls need
+ * none.  All calls on a device share the one scratch array: two calls whose kernels
  * overlap on the GPU (different streams, or different host threads) race on it and give
  * wrong sums, so serialise them.  Nothing in the array has to be cleared between calls:
  * every slot a call reads is first written by that call.

@@ -109,6 +109,9 @@ extern "C" fda_status fda_local_state_linear_noalloc(int device, const float *w,
     if (flags & ~(uint32_t)(FDA_STATE_NORM | FDA_STATE_LINEAR)) return FDA_ERR_INVALID_ARG;
     if (K > FDA_NOALLOC_MAX_WORKERS) return FDA_ERR_UNSUPPORTED;      // beyond the fixed scratch
 
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }
+    if (device >= ndev) return FDA_ERR_INVALID_ARG;                   // no such device
     int prev = -1;
     if (cudaGetDevice(&prev) != cudaSuccess) return FDA_ERR_CUDA;
     if (prev != device && cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return FDA_ERR_CUDA; }

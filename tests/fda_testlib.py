@@ -59,17 +59,28 @@ def check_average(gpu_avg, ora_avg, mean_abs=None):
 
 def check_mean_state(gpu_mean, ora_states, ubar_sq, l, m, d, K, sketch=True):
     """Averaged state S-bar (fp32, one pass on the GPU) against the mean of the oracle's K
-    states.  Scales: the averaged projection and the cells of sk(u-bar) have the size of a
-    random projection / sketch cell of u-bar, so they are compared relative to
-    max(|value|, sqrt(||u-bar||^2/d)) and max(|cell|, sqrt(||u-bar||^2/m)); each of the K drifts
-    entering the sum carries its own fp32 rounding, hence the extra sqrt(K) allowance."""
+    states, at the same relative tolerance as the per-worker states.  Scales: the averaged
+    projection and the cells of sk(u-bar) have the size of a random projection / sketch cell of
+    u-bar, so they are compared relative to max(|value|, sqrt(||u-bar||^2/d)) and
+    max(|cell|, sqrt(||u-bar||^2/m)).  (Measured on B200 over the seven synthetic workloads: the
+    worst cell is off by 1.4e-6 of that scale, the worst projection by 1.0e-7.)  Returns the
+    worst ratios."""
     g = np.asarray(gpu_mean, dtype=np.float64)
     o = np.asarray(ora_states, dtype=np.float64).mean(axis=0)
+    worst = {"norm": abs(g[0] - o[0]) / max(o[0], 1e-300)}
     assert abs(g[0] - o[0]) <= REL * o[0] + 1e-300
-    slack = np.sqrt(K)
     pscale = max(abs(o[1]), np.sqrt(ubar_sq / d), 1e-300)
-    assert abs(g[1] - o[1]) <= REL * slack * pscale
+    worst["proj"] = abs(g[1] - o[1]) / pscale
+    assert worst["proj"] <= REL, worst
     if l > 0 and sketch:
         scale = np.maximum(np.maximum(np.abs(o[2:]), np.sqrt(ubar_sq / m)), 1e-300)
-        err = float(np.max(np.abs(g[2:] - o[2:]) / scale))
-        assert err <= REL * slack, err
+        worst["cell"] = float(np.max(np.abs(g[2:] - o[2:]) / scale))
+        assert worst["cell"] <= REL, worst
+    return worst
+
+
+def mean_estimate_tolerance(ref, ubar_sq):
+    """Tolerance on H of the averaged state: REL on the mean squared norm, and on the estimate of
+    ||u-bar||^2 the bound that follows from cells within REL of max(|cell|, rms cell):
+    |sum of squares - reference| <= 2 REL (sum cell^2 + m rms^2) <= 4 REL max(estimate, ||u-bar||^2)."""
+    return REL * abs(ref["mean_sq"]) + 4 * REL * max(abs(ref["est"]), ubar_sq) + 1e-37

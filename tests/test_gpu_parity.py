@@ -1,9 +1,14 @@
 """GPU parity: libfda (through its C ABI) against the CPU oracle, element by element."""
+import os
+
 import numpy as np
 import pytest
 
 import fda_synth as S
-from fda_testlib import REL, check_average, check_estimate, check_mean_state, check_states, check_trigger
+from fda_testlib import (REL, check_average, check_estimate, check_mean_state, check_states, check_trigger,
+                         mean_estimate_tolerance)
+
+HOST_CORES = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
 
 pytestmark = pytest.mark.gpu
 
@@ -238,8 +243,8 @@ def test_mean_state_matches_mean_of_oracle_states(env, K, d, l, m, misalign):
             e = ctx.fda_combine_estimate(mean.view(1, -1), 1, variant, 0.06, 1e-3, buf).as_dict()
             r = oracle.combine(ora, l, m, variant, 0.06, 1e-3)
             assert abs(e["mean_sq"] - r["mean_sq"]) <= REL * r["mean_sq"]
-            assert abs(e["est"] - r["est"]) <= 4 * REL * np.sqrt(K) * max(r["est"], ubar_sq)
-            tol = REL * r["mean_sq"] + 4 * REL * np.sqrt(K) * max(r["est"], ubar_sq)
+            assert abs(e["est"] - r["est"]) <= 4 * REL * max(r["est"], ubar_sq)
+            tol = mean_estimate_tolerance(r, ubar_sq)
             assert abs(e["H"] - r["H"]) <= tol
             check_trigger(e, r, 1e-3, tol)
 
@@ -392,8 +397,9 @@ def test_average_with_direction_refresh(env):
 
 
 # ----------------------------------------------------------------- the five workloads
-def full_round(env, idx, workers_for_oracle=None, check_avg_ranges=None):
-    """local state -> combine (both variants, every Theta) -> average; oracle beside it."""
+def full_round(env, idx):
+    """local state -> combine (both variants, every Theta) -> averaged state -> average, every worker
+    and every weight against the oracle (all host cores: about 10 s at the two largest workloads)."""
     torch, oracle, F = env
     wl = S.WORKLOADS[idx]
     w_t0 = S.last_global_model(wl)
@@ -401,8 +407,8 @@ def full_round(env, idx, workers_for_oracle=None, check_avg_ranges=None):
     xi = S.unit_direction(wl)
     coeffs = S.hash_coefficients(wl.seed, wl.l)
     d, K = wl.d, wl.K
-    ks = list(range(K)) if workers_for_oracle is None else workers_for_oracle
-    ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, wl.l, wl.m, workers=ks, threads=16)
+    ks = list(range(K))
+    ora = oracle.local_state(wbuf[:, :d], w_t0, xi, coeffs, wl.l, wl.m, threads=HOST_CORES)
     with F.FdaContext(wl.l, wl.m, coeffs, d_max=d, K_max=K) as ctx:
         w = torch.from_numpy(wbuf).cuda()
         w0 = torch.from_numpy(w_t0).cuda()
@@ -422,35 +428,29 @@ def full_round(env, idx, workers_for_oracle=None, check_avg_ranges=None):
                 tol = check_estimate(e, ref, wl.l)
                 check_trigger(e, ref, theta, tol)
                 results[(variant, theta)] = e
-                # ... and, when every worker has an oracle state, end to end as well
-                if workers_for_oracle is None:
-                    ref2 = oracle.combine(ora, wl.l, wl.m, variant, wl.epsilon, float(np.float32(theta)))
-                    tol2 = check_estimate(e, ref2, wl.l)
-                    check_trigger(e, ref2, theta, tol2)
-        # the one-pass averaged state agrees with the average of the K states (linearity)
+                # ... and on the oracle's own states, end to end
+                ref2 = oracle.combine(ora, wl.l, wl.m, variant, wl.epsilon, float(np.float32(theta)))
+                tol2 = check_estimate(e, ref2, wl.l)
+                check_trigger(e, ref2, theta, tol2)
+        # the one-pass averaged state against the mean of the oracle's K states (linearity)
         mean = torch.empty((ctx.state_len,), dtype=torch.float32, device="cuda")
         ctx.fda_mean_state(w[:, :d], w0, xg, ALL, mean)
         torch.cuda.synchronize()
-        gm, avg_states = mean.cpu().numpy().astype(np.float64), got.astype(np.float64).mean(axis=0)
-        ubar_sq = float(results[(F.FDA_VARIANT_SKETCH, wl.thetas[-1])]["est"]) * (1 + wl.epsilon)
-        assert abs(gm[0] - avg_states[0]) <= 2 * REL * avg_states[0]
-        cell_scale = np.maximum(np.abs(avg_states[2:]), np.sqrt(ubar_sq / wl.m))
-        assert np.max(np.abs(gm[2:] - avg_states[2:]) / cell_scale) <= 2 * REL * np.sqrt(K)
+        _, _, ubar_sq = oracle.variance(wbuf[:, :d], w_t0)
+        worst["mean_state"] = check_mean_state(mean.cpu().numpy(), ora, ubar_sq, wl.l, wl.m, d, K)
         e_mean = ctx.fda_combine_estimate(mean.view(1, -1), 1, F.FDA_VARIANT_SKETCH, np.float32(wl.epsilon),
                                           wl.thetas[-1], buf).as_dict()
-        e_ref = results[(F.FDA_VARIANT_SKETCH, wl.thetas[-1])]
-        assert abs(e_mean["H"] - e_ref["H"]) <= 8 * REL * np.sqrt(K) * (abs(e_ref["mean_sq"]) + abs(e_ref["est"]))
-        assert e_mean["trigger"] == e_ref["trigger"]
+        e_ref = oracle.combine(ora, wl.l, wl.m, F.FDA_VARIANT_SKETCH, wl.epsilon, float(np.float32(wl.thetas[-1])))
+        tol_m = mean_estimate_tolerance(e_ref, ubar_sq)
+        assert abs(e_mean["H"] - e_ref["H"]) <= tol_m
+        check_trigger(e_mean, e_ref, wl.thetas[-1], tol_m)
         # average (gated by the last sketch estimate, which fires on every workload)
         e = ctx.fda_combine_estimate(st, K, F.FDA_VARIANT_SKETCH, np.float32(wl.epsilon), wl.thetas[-1], buf)
         assert e.trigger == 1
         ctx.fda_average_models(w[:, :d], w0, buf, F.FDA_AVG_BROADCAST)
         torch.cuda.synchronize()
-        ranges = [(0, d)] if check_avg_ranges is None else check_avg_ranges
         new_w0 = w0.cpu().numpy()
-        mean_abs = float(np.mean(np.abs(new_w0)))
-        for lo, hi in ranges:
-            check_average(new_w0[lo:hi], oracle.average(wbuf[:, :d], lo, hi), mean_abs)
+        check_average(new_w0, oracle.average(wbuf[:, :d]))
         # in-place sync: every row equals the new global model; padding untouched
         for k in (0, K // 2, K - 1):
             assert torch.equal(w[k, :d], w0)
@@ -476,15 +476,11 @@ def test_workload_3_densenet121_full_round(env):
 
 
 def test_workload_4_densenet201_full_size(env):
-    d = S.WORKLOADS[4].d
-    full_round(env, 4, workers_for_oracle=[0, 17, 59],
-               check_avg_ranges=[(0, 50_000), (d // 2 - 3, d // 2 + 40_000), (d - 50_001, d)])
+    full_round(env, 4)
 
 
 def test_workload_5_convnextlarge_full_size(env):
-    d = S.WORKLOADS[5].d
-    full_round(env, 5, workers_for_oracle=[0, 7],
-               check_avg_ranges=[(0, 50_000), (d // 3, d // 3 + 50_000), (d - 50_001, d)])
+    full_round(env, 5)
 
 
 @pytest.mark.parametrize("l,m", [(3, 100), (8, 1000), (5, 250)])

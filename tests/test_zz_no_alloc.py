@@ -1,11 +1,12 @@
-"""fda_local_state_linear_noalloc against fda_local_state.
+"""fda_local_state_linear_noalloc against fda_local_state and against the CPU oracle.
 
 The no-allocation entry point serves callers that cannot create a context because they may
 not call cudaMalloc where they run (a hook inside a training step whose framework allocator
 holds all free memory; an embedder with a fixed memory budget).  Its scratch is one fixed
 array inside the library that keeps whatever the previous call left there, so the check
 runs two calls in a row on different inputs and compares each with the context-based entry
-point, within the tolerance the other parity tests use.  Collected last on purpose.
+point and with the oracle's fp64 norm and projection, within the tolerance the other parity
+tests use.  Collected last on purpose.
 """
 import numpy as np
 import pytest
@@ -48,13 +49,15 @@ def test_no_alloc_entry_point_matches_context_entry_point_twice_in_a_row():
         F.fda_local_state_linear_noalloc(w, w0, xg, flags, states)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before     # the wrapper created no tensor
-        outs.append((states.cpu().numpy().astype(np.float64), w, w0, xg, flags, d))
-    for got, w, w0, xg, flags, d in outs:
-        ref = _reference(F, torch, w, w0, xg, flags)
-        n = ref[:, 0]
-        assert np.all(np.abs(got[:, 0] - n) <= REL * n)
-        scale = np.maximum(np.abs(ref[:, 1]), np.sqrt(n / d))
-        assert np.all(np.abs(got[:, 1] - ref[:, 1]) <= REL * scale)
+        outs.append((states.cpu().numpy().astype(np.float64), w, w0, xg, flags, d, wbuf, w_t0, xi))
+    import oracle
+    for got, w, w0, xg, flags, d, wbuf, w_t0, xi in outs:
+        ora = oracle.local_state(wbuf[:, :d], w_t0, xi if flags & 2 else None, None, 0, 0, threads=4)
+        for ref in (_reference(F, torch, w, w0, xg, flags), ora):
+            n = ref[:, 0]
+            assert np.all(np.abs(got[:, 0] - n) <= REL * n)
+            scale = np.maximum(np.abs(ref[:, 1]), np.sqrt(n / d))
+            assert np.all(np.abs(got[:, 1] - ref[:, 1]) <= REL * scale)
         if not flags & 2:
             assert not got[:, 1].any()
     # beyond the fixed scratch: refused with a clear error, nothing launched
