@@ -165,3 +165,63 @@ def test_last_kernel_names_follow_the_dispatch(env):
         ctx.fda_local_state(w, w0, None, 1 | 4, st)
         assert ctx.fda_debug_last_kernel() in ("k_local_state", "k_local_state_fast")
         torch.cuda.synchronize()
+
+
+def test_sixty_workers_seven_by_five_hundred_run_on_the_list_kernel(env):
+    """The shape of the 20M-parameter workload (K = 60, sketch 7 x 500: lists of about ten entries,
+    fifteen worker groups on nine blocks each), at a size the oracle does in seconds."""
+    run(env, 60, 1_500_007, 7, 500, seed=23, workers=[0, 3, 4, 31, 56, 59])
+    run(env, 58, 700_001, 7, 500, seed=24, flags=1 | 4, workers=[0, 55, 57])      # last group: two workers
+
+
+def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
+    torch, oracle, F = env
+    rng = np.random.default_rng(25)
+    d, K, l, m = 1_000_000, 8, 5, 250
+    coeffs = rand_coeffs(rng, l)
+    w = torch.randn((K, d), device="cuda") * 1e-3
+    w0 = torch.zeros(d, device="cuda")
+    with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+        info = ctx.fda_context_info()
+        assert info["list_kernel"] == 1 and info["tile_indices"] % 1024 == 0 and info["table_bytes"] == 0
+        assert 2.0 * l * d < info["schedule_bytes"] < 3.0 * l * d           # about 2.4 bytes per (row, index)
+        assert info["device_bytes"] >= info["schedule_bytes"] and info["schedule_dropped_bytes"] == 0
+        st = torch.empty((K, ctx.state_len), device="cuda")
+        ctx.fda_local_state(w, w0, None, 1 | 4, st)
+        assert ctx.fda_debug_last_kernel() == GATHER and ctx.fda_context_info()["table_bytes"] == 0
+        mean = torch.empty((ctx.state_len,), device="cuda")
+        ctx.fda_mean_state(w, w0, None, 1 | 4, mean)                         # first use builds the 16-bit table
+        after = ctx.fda_context_info()
+        assert after["table_bytes"] >= 2 * l * d and after["other_lazy_bytes"] >= 4 * d
+        torch.cuda.synchronize()
+        ref = st.cpu().numpy()
+    # a cap below the schedule's size, and no schedule at all: the same states from the other kernels
+    for limit in (1_000_000, -1):
+        with F.FdaContext(l, m, coeffs, d_max=d, K_max=K, schedule_limit_bytes=limit) as ctx:
+            info = ctx.fda_context_info()
+            assert info["list_kernel"] == 0 and info["schedule_bytes"] == 0
+            assert (info["schedule_dropped_bytes"] > 0) == (limit > 0)
+            st = torch.empty((K, ctx.state_len), device="cuda")
+            ctx.fda_local_state(w, w0, None, 1 | 4, st)
+            assert ctx.fda_debug_last_kernel() in ("k_local_state", "k_local_state_fast")
+            torch.cuda.synchronize()
+            got = st.cpu().numpy()
+            n = ref[:, :1]
+            scale = np.maximum(np.abs(ref), np.sqrt(n / m))
+            assert float(np.max(np.abs(got - ref) / scale)) <= 2e-5        # two fp32 paths, each within 1e-5 of the oracle
+
+
+def test_more_worker_groups_than_the_scratch_holds_are_refused(env):
+    """K beyond what the per-block partial sums were sized for: a status, nothing launched."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(26)
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    K, d, l, m = 32 * n_sm + 1, 4096, 2, 16
+    with F.FdaContext(l, m, rand_coeffs(rng, l), d_max=d, K_max=K) as ctx:
+        w = torch.zeros((K, d), device="cuda")
+        st = torch.full((K, ctx.state_len), 7.0, device="cuda")
+        with pytest.raises(F.FdaError) as ei:
+            ctx.fda_local_state(w, torch.zeros(d, device="cuda"), None, 1 | 4, st)
+        assert ei.value.status == 2
+        torch.cuda.synchronize()
+        assert bool((st == 7.0).all())
