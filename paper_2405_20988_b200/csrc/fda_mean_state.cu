@@ -252,9 +252,9 @@ __global__ void __launch_bounds__(32 * FDA_MAX_ROWS, 1) k_sketch_vector_rows(con
         const float v0 = flip(a.x, (h.x << 16) & 0x80000000u), v1 = flip(a.y, h.x & 0x80000000u);
         const float v2 = flip(a.z, (h.y << 16) & 0x80000000u), v3 = flip(a.w, h.y & 0x80000000u);
         const float o0 = lds_f32(a0), o1 = lds_f32(a1), o2 = lds_f32(a2), o3 = lds_f32(a3);
-        // equal cells among the four: every store to such a cell carries the sum of all of them, so
-        // the result does not depend on the order in which the stores land (two stores of one
-        // thread to one shared address were observed to land out of program order on B200)
+        // equal cells among the four: the four loads above are issued before the four stores below,
+        // so two updates of one cell would both start from the old value and one would be lost
+        // whatever the order of the stores; every store to such a cell carries the sum of all of them
         const bool e01 = a0 == a1, e02 = a0 == a2, e03 = a0 == a3, e12 = a1 == a2, e13 = a1 == a3, e23 = a2 == a3;
         const float t0 = v0 + (e01 ? v1 : 0.f) + (e02 ? v2 : 0.f) + (e03 ? v3 : 0.f);
         const float t1 = v1 + (e01 ? v0 : 0.f) + (e12 ? v2 : 0.f) + (e13 ? v3 : 0.f);
