@@ -11,13 +11,17 @@
 // to be cut into pieces are added atomically).  One update costs one 4-byte shared-memory read.
 //
 // A block serves a group of 4 workers and a strided set of tiles, with two kinds of warps:
-//   producers  8 warps.  A thread owns four consecutive indices of a 1024-index batch: it loads
-//              the four workers' values and w_t0 (xi) with 128-bit loads, two batches in
-//              flight per thread (the registers are the landing zone: nothing else is staged;
-//              32-bit loads could not keep enough bytes in flight), subtracts, adds up ||u||^2
-//              and <xi,u> (fp32 within a tile, fp64 across tiles) and stores the four drifts of
-//              an index as one 16-byte row of the tile: ut[index][4];
-//   walkers    20 warps.  They take the tile's items (32 lists, one per lane) from a counter,
+//   producers  8 warps (4 for sketches of 7 or more rows).  A thread owns four consecutive indices
+//              of a batch (1024 indices with 8 warps): it loads the four workers' values and w_t0
+//              (xi) with 128-bit loads into registers (the landing zone: nothing else is staged),
+//              subtracts, adds up ||u||^2 and <xi,u> (fp32 within a tile, fp64 across tiles) and
+//              stores the four drifts of an index as one 16-byte row of the tile: ut[index][4].
+//              The next batch is asked for as soon as the registers are free.  Measured on B200:
+//              what a block streams from memory grows with the number of warps that have loads
+//              in flight (4.6 TB/s with 8 warps per SM, 6.5 with 16, 7.0 with 24), not with the
+//              loads a warp has in flight; deeper software pipelines here changed nothing, and
+//              32-bit loads ran at a quarter of the speed;
+//   walkers    20 warps (24).  They take the tile's items (32 lists, one per lane) from a counter,
 //              longest first; per step a lane loads one 16-bit entry's row with a 128-bit load
 //              (the schedule orders the entries so that the eight lanes of a pass through
 //              shared memory hit eight different bank groups) and adds it with the entry's
@@ -33,18 +37,8 @@
 namespace {
 
 constexpr int GW = kListWorkers;
-#ifndef FDA_PW
-#define FDA_PW 8
-#define FDA_WW 20
-#define FDA_DEPTH 1
-#endif
-constexpr int kProducerWarps = FDA_PW;
-constexpr int kWalkerWarps = FDA_WW;
-constexpr int kThreads = (kProducerWarps + kWalkerWarps) * 32;
-constexpr int kDepth = FDA_DEPTH;                      // batches a producer thread keeps in flight
 constexpr int kChunksAhead = 8;                // entry chunks (four steps each) a walker loads before it walks them
-constexpr int kBatch = kProducerWarps * 32 * 4;   // a batch is four consecutive indices per producer thread
-static_assert(kProducerWarps <= 16 && kListBatch % kBatch == 0, "tiles are whole batches; the fp64 sums have room for 16 producer warps");
+constexpr int kMaxProducerWarps = 16;          // the fp64 sums in shared memory have room for that many
 
 struct ListParams {
     const float *w, *w_t0, *xi;
@@ -64,9 +58,10 @@ struct ListParams {
     double *part_np;                 // [block][GW][2]
 };
 
+template <int THREADS>
 __device__ __forceinline__ void block_barrier()
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
 }
 
 // Loads and stores of the producers as volatile statements: the compiler keeps them in program
@@ -145,9 +140,16 @@ __device__ __forceinline__ void gather_hi(uint32_t w, uint32_t base, unsigned lo
 //   [576, ..) two item tables (tab_bytes each): the head of a tile's schedule record
 //   then      bins[l*m][4]
 //   then      ut[2][T + 8][4]   (drift tiles, index-major; eight zero rows behind each)
-template <bool LINEAR>
-__global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListParams p)
+// PW producer warps and WW walker warps: the split that is fastest depends on how much walking a
+// loaded index pays for (l updates per worker).
+template <bool LINEAR, int PW, int WW>
+__global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const ListParams p)
 {
+    constexpr int kProducerWarps = PW;
+    constexpr int kThreads = (PW + WW) * 32;
+    constexpr int kBatch = PW * 32 * 4;                       // a batch is four consecutive indices per producer thread
+    constexpr int kDepth = 1;                                 // batches a producer thread keeps in flight
+    static_assert(PW <= kMaxProducerWarps, "the fp64 sums have room for kMaxProducerWarps warps");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = (int)blockIdx.x % p.groups, c = (int)blockIdx.x / p.groups;
@@ -293,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
                     off1 = load_u64(p.sched_off + t2 + 1);
                 }
                 prefetch_tile(n_c + 2);
-                block_barrier();
+                block_barrier<kThreads>();
                 b_c = 0;
                 ++n_c;
             }
@@ -309,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
     } else {
         // =============================== walkers ===============================
         for (int64_t n = 0; n < n_tiles; ++n) {
-            block_barrier();                                   // tile n is stored, tile n - 1 is walked
+            block_barrier<kThreads>();                                   // tile n is stored, tile n - 1 is walked
             const int buf = (int)(n & 1);
             const unsigned char *rec = p.sched + p.sched_off[c + n * p.cpg];
             const uint32_t *tab = reinterpret_cast<const uint32_t *>(smem_raw + tab_off + (size_t)buf * p.tab_bytes);
@@ -367,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_local_state_gather(const ListPa
             }
         }
     }
-    block_barrier();                                           // the last tile is walked
+    block_barrier<kThreads>();                                           // the last tile is walked
 
     // ---- flush: bins -> this block's partial sketch ----
     {
@@ -427,6 +429,18 @@ __global__ void k_finalize_gather(const ListParams p, int blocks, uint32_t flags
     }
 }
 
+template <int PW, int WW>
+cudaError_t launch_lists(ListParams &p, int blocks, size_t smem, int smem_optin, cudaStream_t s)
+{
+    if (p.T % (PW * 128) != 0 || PW * 32 * 16 < p.tab_bytes) return cudaErrorNotSupported;
+    p.nb = p.T / (PW * 128);
+    auto kern = p.have_xi ? k_local_state_gather<true, PW, WW> : k_local_state_gather<false, PW, WW>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    if (e != cudaSuccess) return e;
+    kern<<<blocks, (PW + WW) * 32, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 // Returns cudaErrorNotSupported when the request does not fit this path (the caller then uses
@@ -443,8 +457,7 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     p.K = K; p.d = d; p.have_xi = xi_used != nullptr;
     p.vec = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) && (row_stride % 4 == 0);
     p.l = ctx->l; p.m = ctx->m;
-    p.T = ctx->sched_T; p.nb = p.T / kBatch;
-    if (p.T % kBatch != 0) return cudaErrorNotSupported;
+    p.T = ctx->sched_T;
     p.sched = ctx->sched; p.sched_off = ctx->sched_off;
     p.part_sk = ctx->part_sk; p.part_np = ctx->part_np;
     p.tiles = (d + p.T - 1) / p.T;
@@ -461,13 +474,14 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
         (size_t)blocks * GW * 2 > ctx->part_np_doubles)
         return cudaErrorNotSupported;
     const size_t smem = fda_list_smem_bytes(p.l, p.m, p.T, ctx->sched_ni_max);
-    if (smem > (size_t)ctx->smem_optin || kProducerWarps * 32 * 16 < p.tab_bytes) return cudaErrorNotSupported;
+    if (smem > (size_t)ctx->smem_optin) return cudaErrorNotSupported;
 
-    auto kern = xi_used ? k_local_state_gather<true> : k_local_state_gather<false>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin);
-    if (e != cudaSuccess) return e;
-    kern<<<blocks, kThreads, smem, s>>>(p);
-    e = cudaGetLastError();
+    // 8 producer + 20 walker warps, or 4 + 24 when a loaded index pays for more walking.  Measured:
+    // 7 x 500, K = 60, d = 20M: 3.34 ms with 4 + 24 against 3.71 ms with 8 + 20; 5 x 250, K = 8,
+    // d = 198M: 3.49 against 2.49 ms; 5 x 250, K = 30, d = 7M: 0.535 against 0.387 ms.
+    cudaError_t e;
+    if (ctx->l >= 7) e = launch_lists<4, 24>(p, blocks, smem, ctx->smem_optin, s);
+    else e = launch_lists<8, 20>(p, blocks, smem, ctx->smem_optin, s);
     if (e != cudaSuccess) return e;
     const int64_t total = (int64_t)p.groups * (2 + ctx->lm) * GW * 4;
     int fb = (int)((total + 255) / 256);
