@@ -14,7 +14,8 @@
 //   * so the lists are grouped by eight (an octet): starting from the longest list left, the
 //     builder adds the longest lists whose indices keep every residue class mod 8 of the octet
 //     at or below the length of the first one (a class with c indices needs c passes whatever
-//     the order).  The entries of an octet are then ordered by decomposing the bipartite
+//     the order), counting a list whose cell shares a bank group with a cell already in the
+//     octet (a conflict when the sums are flushed) as two entries shorter.  The entries of an octet are then ordered by decomposing the bipartite
 //     multigraph (lists x residue classes, one edge per index, made regular with padding edges)
 //     into perfect matchings: in every step each lane reads a different residue class, and a
 //     lane with nothing left reads a zero row of a class nobody else reads;
@@ -269,7 +270,9 @@ __global__ void __launch_bounds__(kBT) k_build_schedule(const SchedParams p)
                             uint32_t k;
                             if (mx <= L) {
                                 const uint32_t conflict = (cellmask >> (ls_cell[cand] & 7)) & 1u;
-                                k = ((uint32_t)(L - ls_len[cand]) << 23) | (conflict << 22) |
+                                // a flush conflict (two cells of the octet in one bank group) costs about
+                                // as much as two idle steps of a lane
+                                k = ((uint32_t)(L - ls_len[cand] + 2 * (int)conflict) << 23) |
                                     ((uint32_t)min(sq, 0xffff) << 6) | (uint32_t)slot;
                             } else {
                                 k = 0x80000000u | ((uint32_t)min(mx, 0x3ff) << 21) |
