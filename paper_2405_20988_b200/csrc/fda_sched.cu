@@ -42,6 +42,11 @@ constexpr int kBT = 256;                  // threads of a builder block
 constexpr int ML = kListMaxLen;
 constexpr int NRES = kListOct;            // residue classes = lanes per shared-memory pass
 constexpr int kWindow = 64;               // candidates looked at for every place in an octet
+#ifndef FDA_SPREAD
+#define FDA_SPREAD 8
+#endif
+constexpr int kMatchBytes = 304;          // shared memory of the thread that orders an octet's entries
+constexpr int kSpread = FDA_SPREAD;       // every kSpread-th thread of the block orders the entries of an octet
 
 struct SchedParams {
     const uint64_t *coeffs;
@@ -355,7 +360,9 @@ __global__ void __launch_bounds__(kBT) k_build_schedule(const SchedParams p)
             }
             // ---- entries: one thread per octet place of the row's items ----
             uint16_t *ent = reinterpret_cast<uint16_t *>(rec + ent_off);
-            for (int pos = tid; pos < 4 * ni_row; pos += kBT) {
+            // (spread over the warps of the block: the matching is serial code on private tables,
+            // and threads of one warp would run its data-dependent paths one after the other)
+            for (int pos = tid / kSpread; (tid % kSpread) == 0 && pos < 4 * ni_row; pos += kBT / kSpread) {
                 const int q = pos / 4, lane0 = (pos % 4) * NRES;
                 const int steps = (int)it_steps[item0 + q];
                 const int padded = (steps + 3) & ~3;
@@ -367,34 +374,38 @@ __global__ void __launch_bounds__(kBT) k_build_schedule(const SchedParams p)
                 if (pos < no) {
                     const int o = oc_order[pos];
                     delta = oc_cost[o];
-                    // C: indices of list s in class r; D: padding edges that make the graph regular
-                    unsigned short C[NRES * NRES], D[NRES * NRES], cur[NRES * NRES];
-                    int defL[NRES], defR[NRES];
-#pragma unroll
-                    for (int r = 0; r < NRES; ++r) defR[r] = delta;
+                    // C: indices of list s in class r; D: padding edges that make the graph regular.
+                    // The tables live in shared memory (the hash words of the row are no longer
+                    // needed): as private arrays they spill to local memory, which the block's
+                    // shared-memory footprint leaves almost no L1 for.
+                    unsigned char *mt = reinterpret_cast<unsigned char *>(key) + (size_t)pos * kMatchBytes;
+                    unsigned char *C = mt, *D = mt + 64;
+                    unsigned short *cur = reinterpret_cast<unsigned short *>(mt + 128);
+                    signed char *match = reinterpret_cast<signed char *>(mt + 256);
+                    signed char *matchR = match + 8, *prevS = match + 16, *queue = match + 24;
+                    unsigned char *defL = mt + 288, *defR = mt + 296;
+                    for (int r = 0; r < NRES; ++r) defR[r] = (unsigned char)delta;
                     for (int s = 0; s < NRES; ++s) {
                         const int li = oc_list[8 * o + s];
                         int a0 = li != 0xffff ? ls_start[li] : 0, len = 0;
                         for (int r = 0; r < NRES; ++r) {
                             const int v = li != 0xffff ? ls_res[8 * li + r] : 0;
-                            C[s * NRES + r] = (unsigned short)v;
+                            C[s * NRES + r] = (unsigned char)v;
                             D[s * NRES + r] = 0;
                             cur[s * NRES + r] = (unsigned short)a0;
                             a0 += v;
                             len += v;
-                            defR[r] -= v;
+                            defR[r] = (unsigned char)(defR[r] - v);
                         }
-                        defL[s] = delta - len;
+                        defL[s] = (unsigned char)(delta - len);
                     }
                     for (int s = 0, r = 0; s < NRES && r < NRES;) {
-                        const int x = min(defL[s], defR[r]);
-                        D[s * NRES + r] = (unsigned short)(D[s * NRES + r] + x);
-                        defL[s] -= x;
-                        defR[r] -= x;
+                        const int x = min((int)defL[s], (int)defR[r]);
+                        D[s * NRES + r] = (unsigned char)(D[s * NRES + r] + x);
+                        defL[s] = (unsigned char)(defL[s] - x);
+                        defR[r] = (unsigned char)(defR[r] - x);
                         if (defL[s] == 0) ++s; else ++r;
                     }
-                    int match[NRES], matchR[NRES];
-#pragma unroll
                     for (int s = 0; s < NRES; ++s) match[s] = -1;
                     for (int t = 0; t < delta; ++t) {
                         // keep the edges of the last matching that still exist, complete it with
@@ -402,13 +413,13 @@ __global__ void __launch_bounds__(kBT) k_build_schedule(const SchedParams p)
                         for (int r = 0; r < NRES; ++r) matchR[r] = -1;
                         for (int s = 0; s < NRES; ++s) {
                             const int r = match[s];
-                            if (r >= 0 && (C[s * NRES + r] | D[s * NRES + r]) != 0) matchR[r] = s; else match[s] = -1;
+                            if (r >= 0 && (C[s * NRES + r] | D[s * NRES + r]) != 0) matchR[r] = (signed char)s; else match[s] = -1;
                         }
                         for (int s0 = 0; s0 < NRES; ++s0) {
                             if (match[s0] >= 0) continue;
-                            int prevS[NRES], queue[NRES], qh = 0, qt = 0;
+                            int qh = 0, qt = 0;
                             unsigned vis = 0;
-                            queue[qt++] = s0;
+                            queue[qt++] = (signed char)s0;
                             bool done = false;
                             while (qh < qt && !done) {
                                 const int s = queue[qh++];
@@ -416,14 +427,14 @@ __global__ void __launch_bounds__(kBT) k_build_schedule(const SchedParams p)
                                     if ((vis >> r) & 1u) continue;
                                     if ((C[s * NRES + r] | D[s * NRES + r]) == 0) continue;
                                     vis |= 1u << r;
-                                    prevS[r] = s;
+                                    prevS[r] = (signed char)s;
                                     if (matchR[r] < 0) {
                                         int rc = r;
                                         for (;;) {
                                             const int sp = prevS[rc];
                                             const int nr = match[sp];
-                                            match[sp] = rc;
-                                            matchR[rc] = sp;
+                                            match[sp] = (signed char)rc;
+                                            matchR[rc] = (signed char)sp;
                                             if (sp == s0) break;
                                             rc = nr;
                                         }
@@ -520,6 +531,8 @@ cudaError_t fda_build_list_schedule(fda_ctx *ctx, cudaStream_t s)
     p.ni_row_max = (p.nl_max + kListSlots - 1) / kListSlots;
     const size_t bsmem = build_smem(p.l, p.m, T, p.nl_max, p.no_max, p.ni_row_max);
     if (bsmem > (size_t)ctx->smem_optin) return cudaSuccess;
+    // the matching tables of a row's octets reuse the two arrays of hash words (8 bytes per index)
+    if ((size_t)4 * p.ni_row_max * kMatchBytes > 2 * sizeof(uint32_t) * (size_t)T) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(k_build_schedule<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bsmem);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_build_schedule<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bsmem);
