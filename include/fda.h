@@ -8,8 +8,8 @@
  *   fda_combine_estimate -> S-bar = mean_k S^(k), H(S-bar), trigger = (H > Theta)
  *   fda_average_models   -> w^(k) := w-bar = mean_k w^(k)  (and w_t0 := w-bar) if triggered
  *
- * which are lines 6-9 of Algorithm 1 of the FDA paper (Section 3) with the two AllReduce
- * steps replaced by reductions over rows in device memory.
+ * which are the monitoring and synchronisation steps of Algorithm 1 of the FDA paper (Section 3)
+ * with the two AllReduce steps replaced by reductions over rows in device memory.
  *
  * Conventions
  *   - plain C ABI; every function returns an fda_status and never throws or aborts;
@@ -91,8 +91,9 @@ typedef struct {
  *     and sketch requests are then served by the slower plain-load kernels, when it would take
  *     more than a third of the free device memory (see fda_create_limited for another cap);
  *   - lazily, by the first call that needs them: a 16-bit hash table of 2*l bytes per index
- *     (sketch requests without a schedule, fda_mean_state), d_max floats (fda_mean_state),
- *     K_max*d_max floats of staging (fda_round_host).
+ *     (sketch requests on a context without a schedule), d_max floats (fda_mean_state with
+ *     more than 2*l workers, or without a schedule), K_max*d_max floats of staging
+ *     (fda_round_host).
  * Blocking: allocates, builds the schedule, synchronises the device.
  * Errors: INVALID_ARG (out == NULL, l < 0 or > FDA_MAX_ROWS, m < 1 or > 32768 with l > 0,
  * d_max < 1 or >= 2^31, K_max < 1, coefficient out of range), UNSUPPORTED (l*m too large
@@ -153,18 +154,21 @@ fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int
  * state_len floats) = ( (1/K) sum_k ||u^(k)||^2, (1/K) sum_k <xi,u^(k)>, sk(u-bar) ) with
  * u-bar = (1/K) sum_k u^(k).  By the linearity of the sketch (Section 3.1, property (a); the
  * "(lin.)" step in the proof of Theorem 1) sk(u-bar) equals the average of the K worker
- * sketches that Algorithm 1 line 7 forms, so fda_combine_estimate(ctx, mean_state, K = 1, ...)
+ * sketches that Algorithm 1 forms when it averages the states, so fda_combine_estimate(ctx, mean_state, K = 1, ...)
  * yields the same H and trigger as the per-worker route, with l instead of K*l bin updates
- * per index.  Arguments and errors as fda_local_state; mean_state is state_len floats.  The
- * first call on a context allocates d_max floats of scratch for the average drift (NOMEM if
- * that fails).
+ * per index.  Arguments and errors as fda_local_state; mean_state is state_len floats.  On a
+ * context with a list schedule the cells come from the list kernel: in one pass over the K rows
+ * for K <= 2*l, else from the vector of averaged drifts that a first pass leaves in device
+ * memory; that vector (d_max floats) is allocated by the first call that needs it (NOMEM if that
+ * fails), and so is the 16-bit hash table on a context without a schedule.
  */
 fda_status fda_mean_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                           const float *w_t0, const float *xi, uint32_t flags, float *mean_state,
                           void *stream);
 
 /*
- * Average the K states and evaluate the variance over-estimate (Algorithm 1 lines 7-8).
+ * Average the K states and evaluate the variance over-estimate (Algorithm 1: the state average and
+ * the variance test).
  *   FDA_VARIANT_SKETCH: H = S-bar[0] - median_i ||row_i(S-bar sketch)||^2 / (1 + epsilon)
  *                       (Theorem 1; the median of an even number of rows is the mean of
  *                       the two middle values);
@@ -183,8 +187,8 @@ fda_status fda_combine_estimate(fda_ctx *ctx, const float *states, int K, int va
 
 /*
  * Synchronise: w-bar[j] = (1/K) sum_k w^(k)[j] (fp32, summed in the order k = 0..K-1), then
- * w_t0 := w-bar and, with FDA_AVG_BROADCAST, every w^(k) := w-bar in place (Section 3,
- * "Workers synchronize by executing AllReduce"; Algorithm 1 line 9).
+ * w_t0 := w-bar and, with FDA_AVG_BROADCAST, every w^(k) := w-bar in place (Section 3: the
+ * workers synchronise with an AllReduce of their models; the synchronisation step of Algorithm 1).
  *   est_dev     DEVICE fda_estimate whose `trigger` gates the whole operation on the
  *               device (nothing is read or written when it is 0); NULL or
  *               FDA_AVG_UNCONDITIONAL averages always.
@@ -271,11 +275,14 @@ fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_hos
                               int64_t *info);
 
 /*
- * Name of the kernel that served the context's last fda_local_state call (the paper has no
- * counterpart): "k_local_state_gather" (sketch pass over per-cell index lists: every sketch request
+ * Name of the kernel that served the context's last fda_local_state or fda_mean_state call (the
+ * paper has no counterpart): "k_local_state_gather" (sketch pass over per-cell index lists: every sketch request
  * on a context that holds a list schedule), "k_local_state_linear" (no sketch requested),
  * "k_local_state_fast" / "k_local_state" (sketch requests without a schedule: aligned rows with 5
- * or 7 sketch rows / everything else), or "" before the first call.  The string is static;
+ * or 7 sketch rows / everything else); for fda_mean_state "k_local_state_gather(mean)" (one pass on
+ * the list kernel), "k_mean_model + k_local_state_gather(mean)" (averaged drifts, then the list
+ * kernel on them), "k_mean_model + k_sketch_vector" (no schedule) or "k_mean_model" (no sketch
+ * requested); "" before the first call.  The string is static;
  * ctx == NULL gives "".  Tests and the benchmark use it to say which kernel a number belongs to.
  */
 const char *fda_debug_last_kernel(const fda_ctx *ctx);

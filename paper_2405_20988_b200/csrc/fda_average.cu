@@ -1,5 +1,5 @@
-// K-way model average (Section 3: "Workers synchronize by executing AllReduce", Algorithm 1
-// line 9): w-bar = (1/K) sum_k w^(k), written to w_t0 and, when broadcasting, to every row.
+// K-way model average (Section 3: the workers synchronise with an AllReduce of their models,
+// the synchronisation step of Algorithm 1): w-bar = (1/K) sum_k w^(k), written to w_t0 and, when broadcasting, to every row.
 // Bandwidth-bound streaming kernel; the whole launch is predicated on the trigger word of
 // the device-side estimate so that no host round trip is needed between the two calls.
 #include "fda_internal.h"

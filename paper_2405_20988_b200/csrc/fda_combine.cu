@@ -1,5 +1,5 @@
 // Combine step: average state, row norms of the averaged sketch, median, H, trigger
-// (Algorithm 1 lines 7-8; Theorem 1 for SketchFDA, Theorem 2 for LinearFDA).
+// (Algorithm 1: the state average and the variance test; Theorem 1 for SketchFDA, Theorem 2 for LinearFDA).
 //
 // One block per sketch row plus one for the two scalar entries, so that the K x (2 + l*m) reads
 // of a large state table are spread over several SMs; the block that finishes last (a ticket

@@ -75,7 +75,7 @@ struct fda_ctx {
     fda_estimate *stage_est = nullptr;
     int64_t stage_stride = 0;
     uint64_t coeffs_host[6 * FDA_MAX_ROWS] = {0};
-    const char *last_ls_kernel = "";   // which kernel served the last fda_local_state
+    const char *last_ls_kernel = "";   // which kernel served the last fda_local_state / fda_mean_state
     std::string err;
 };
 
@@ -92,6 +92,11 @@ cudaError_t fda_build_list_schedule(fda_ctx *ctx, cudaStream_t s);   // allocate
 cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);
+cudaError_t fda_launch_mean_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                         int64_t d, const float *w_t0, const float *xi,
+                                         uint32_t flags, float *mean_state, cudaStream_t s);
+cudaError_t fda_launch_mean_sketch_gather(fda_ctx *ctx, const float *mean_drift, int K, int64_t d, bool have_xi,
+                                          uint32_t flags, int np_blocks, float *mean_state, cudaStream_t s);
 cudaError_t fda_launch_local_state_linear(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
                                           int64_t d, const float *w_t0, const float *xi,
                                           uint32_t flags, float *states, cudaStream_t s);

@@ -56,6 +56,8 @@ struct ListParams {
     const uint64_t *sched_off;
     float *part_sk;                  // [block][cell][GW]
     double *part_np;                 // [block][GW][2]
+    int base_zero;                   // averaged state only: the rows are drifts already (no w_t0 to subtract)
+    int sketch_only;                 // averaged state only: leave part_np alone
 };
 
 template <int THREADS>
@@ -136,20 +138,24 @@ __device__ __forceinline__ void gather_hi(uint32_t w, uint32_t base, unsigned lo
 
 // Shared-memory plan (bytes from the start of dynamic shared memory):
 //   [0, 8)    item counters of the two tile buffers
-//   [64, 576) sums[producer warp][worker][2] (fp64): ||u||^2 and <xi,u> over the tiles so far
-//   [576, ..) two item tables (tab_bytes each): the head of a tile's schedule record
+//   [64, 1088) sums[producer warp][worker][2] (fp64): ||u||^2 and <xi,u> over the tiles so far
+//   [1088, ..) two item tables (tab_bytes each): the head of a tile's schedule record
 //   then      bins[l*m][4]
 //   then      ut[2][T + 8][4]   (drift tiles, index-major; eight zero rows behind each)
 // PW producer warps and WW walker warps: the split that is fastest depends on how much walking a
 // loaded index pays for (l updates per worker).
-template <bool LINEAR, int PW, int WW>
+// MEAN (the averaged state of fda_mean_state; by linearity, Section 3.1 (a), the sketch of the
+// mean drift): one block group serves all K workers, the first column of a row of the tile holds
+// the sum of all workers' drifts and the other three are zero, so the walk costs l updates per
+// index instead of K*l; the sums are divided by K at the end.
+template <bool LINEAR, bool MEAN, int PW, int WW>
 __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const ListParams p)
 {
     constexpr int kProducerWarps = PW;
     constexpr int kThreads = (PW + WW) * 32;
     constexpr int kBatch = PW * 32 * 4;                       // a batch is four consecutive indices per producer thread
     constexpr int kDepth = 1;                                 // batches a producer thread keeps in flight
-    static_assert(PW <= kMaxProducerWarps, "the fp64 sums have room for kMaxProducerWarps warps");
+    static_assert(PW <= (MEAN ? 4 * kMaxProducerWarps : kMaxProducerWarps), "room for the fp64 sums of the producer warps");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = (int)blockIdx.x % p.groups, c = (int)blockIdx.x / p.groups;
@@ -170,7 +176,7 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
         reinterpret_cast<float *>(smem_raw + ut_off + (size_t)b * ut_bytes)[T * GW + r] = 0.f;
     }
     if (tid < 2) ctr[tid] = 0;
-    if (tid < kProducerWarps * GW * 2) sums[tid] = 0.0;
+    if (tid < kMaxProducerWarps * GW * 2) sums[tid] = 0.0;
     __syncthreads();
 
     const int64_t n_tiles = p.tiles > c ? (p.tiles - c + p.cpg - 1) / p.cpg : 0;
@@ -178,35 +184,28 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
     if (warp < kProducerWarps) {
         // =============================== producers ===============================
         const int pt = tid;                                   // quad of indices inside a batch
-        // rows of the group; workers past K alias the group's first row (their sums are computed
-        // and never written out), so the loop below needs no per-worker predicate
-        const float *wbase = p.w + (size_t)(g * GW) * (size_t)p.row_stride;
-        int64_t roff[GW];
-#pragma unroll
-        for (int k = 0; k < GW; ++k) roff[k] = g * GW + k < p.K ? (int64_t)k * p.row_stride : 0;
-        float4 wv[kDepth][GW], w0v[kDepth], xv[kDepth];       // four consecutive indices each
+        const bool vec_in = p.vec != 0;
         float nf[GW], pf[GW];
 #pragma unroll
         for (int k = 0; k < GW; ++k) { nf[k] = 0.f; pf[k] = 0.f; }
-        int64_t n_i = 0, n_c = 0;                             // tile being loaded / stored
-        int b_i = 0, b_c = 0;                                 // batch inside it
-        int64_t j_i = (int64_t)c * T + 4 * pt;                // first index of this thread's next loads
-        int64_t end_i = (int64_t)(c + 1) * T;                 // end of the tile they belong to
-        const int64_t wrap = (int64_t)(p.cpg - 1) * T;        // from the end of a tile to this block's next one
-        const bool vec_in = p.vec != 0;
+        // rows of the group (MEAN: the group is all K workers, g = 0)
+        const float *wbase = p.w + (size_t)(g * GW) * (size_t)p.row_stride;
 
         // The rows of a tile two tiles ahead of the one being stored, into L2 (one bulk prefetch per
         // worker row, w_t0 and xi): the producers' loads then find their data in L2.
         auto prefetch_tile = [&](int64_t n) {
-            if (n >= n_tiles || !vec_in || pt >= GW + 2) return;
+            const int n_rows = MEAN ? p.K : GW;
+            if (n >= n_tiles || !vec_in || pt >= n_rows + 2) return;
             const int64_t j = (c + n * p.cpg) * (int64_t)T;
             int64_t cnt = p.d - j;
             if (cnt > T) cnt = T;
             const uint32_t bytes = (uint32_t)(cnt * 4) & ~15u;
-            const float *src = pt < GW ? (g * GW + pt < p.K ? wbase + (int64_t)pt * p.row_stride + j : nullptr)
-                                       : (pt == GW ? p.w_t0 + j : (LINEAR ? p.xi + j : nullptr));
-            if (src && bytes)
-                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+            for (int r = pt; r < n_rows + 2; r += kProducerWarps * 32) {
+                const float *src = r < n_rows ? (g * GW + r < p.K ? wbase + (int64_t)r * p.row_stride + j : nullptr)
+                                              : (r == n_rows ? (MEAN && p.base_zero ? nullptr : p.w_t0 + j) : (LINEAR ? p.xi + j : nullptr));
+                if (src && bytes)
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+            }
         };
         prefetch_tile(0);
         prefetch_tile(1);
@@ -216,54 +215,24 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
         unsigned long long off0 = load_u64(p.sched_off + c), off1 = load_u64(p.sched_off + c + 1);
         if (pt * 16 < p.tab_bytes) tabv = load_u4(p.sched + off0 + pt * 16);
         if (n_tiles > 1) { off0 = load_u64(p.sched_off + c + p.cpg); off1 = load_u64(p.sched_off + c + p.cpg + 1); }
-        auto issue = [&](int slot) {
-            if (n_i < n_tiles) {
-                const float *q = wbase + j_i;
-                if (vec_in && end_i <= p.d) {                 // a whole tile of aligned rows: 128-bit loads
+
+        // ---- tile n of this block is stored: its sums, its item table, its counter, then the hand-over ----
+        auto end_of_tile = [&](int64_t n) {
+            const int buf = (int)(n & 1);
+            // (fp32 within the tile: a thread's few indices, then the warp's tree; fp64 across tiles)
+            if (MEAN) {
+                float a = nf[0], bq = LINEAR ? pf[0] : 0.f;
 #pragma unroll
-                    for (int k = 0; k < GW; ++k) wv[slot][k] = load4_stream(q + roff[k]);
-                    w0v[slot] = load4_keep(p.w_t0 + j_i);
-                    if (LINEAR) xv[slot] = load4_keep(p.xi + j_i);
-                } else {                                      // the last tile of the model, or unaligned rows
-                    const int64_t left = p.d - j_i;
-                    const int n = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
-                    const bool vec = vec_in && n == 4;
-#pragma unroll
-                    for (int k = 0; k < GW; ++k) wv[slot][k] = load_quad<true>(q + roff[k], vec, n);
-                    w0v[slot] = load_quad<false>(p.w_t0 + j_i, vec, n);
-                    if (LINEAR) xv[slot] = load_quad<false>(p.xi + j_i, vec, n);
+                for (int off = 16; off > 0; off >>= 1) {
+                    a += __shfl_xor_sync(0xffffffffu, a, off);
+                    if (LINEAR) bq += __shfl_xor_sync(0xffffffffu, bq, off);
                 }
-                j_i += kBatch;
-                if (++b_i == p.nb) { b_i = 0; ++n_i; j_i += wrap; end_i += wrap + T; }
-            }
-        };
-        auto consume = [&](int slot) {
-            const int buf = (int)(n_c & 1);
-            // rows 4*pt .. 4*pt+3 of the batch; row r is stored at r ^ ((r >> 3) & 3), so that the
-            // eight lanes of a store pass hit eight different bank groups (the schedule's entries
-            // hold the swizzled row)
-            const uint32_t r0 = (uint32_t)(b_c * kBatch + 4 * pt);
-            const uint32_t dst0 = smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 16u;
-            const uint32_t sw = (r0 >> 3) & 3u;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float w0 = comp(w0v[slot], q);
-                const float u0 = comp(wv[slot][0], q) - w0;
-                const float u1 = comp(wv[slot][1], q) - w0;
-                const float u2 = comp(wv[slot][2], q) - w0;
-                const float u3 = comp(wv[slot][3], q) - w0;
-                nf[0] = fmaf(u0, u0, nf[0]); nf[1] = fmaf(u1, u1, nf[1]);
-                nf[2] = fmaf(u2, u2, nf[2]); nf[3] = fmaf(u3, u3, nf[3]);
-                if (LINEAR) {
-                    const float xq = comp(xv[slot], q);
-                    pf[0] = fmaf(xq, u0, pf[0]); pf[1] = fmaf(xq, u1, pf[1]);
-                    pf[2] = fmaf(xq, u2, pf[2]); pf[3] = fmaf(xq, u3, pf[3]);
+                if (lane == 0) {
+                    sums[warp * 2 + 0] += (double)a;
+                    if (LINEAR) sums[warp * 2 + 1] += (double)bq;
                 }
-                store_row(dst0 + (((uint32_t)q ^ sw) << 4), u0, u1, u2, u3);
-            }
-            if (++b_c == p.nb) {
-                // ---- the tile is stored: its item table, its counter, then the hand-over ----
-                // (fp32 within the tile: a thread's few indices, then the warp's tree; fp64 across tiles)
+                nf[0] = 0.f; pf[0] = 0.f;
+            } else {
 #pragma unroll
                 for (int k = 0; k < GW; ++k) {
                     float a = nf[k], bq = LINEAR ? pf[k] : 0.f;
@@ -278,34 +247,173 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
                     }
                     nf[k] = 0.f; pf[k] = 0.f;
                 }
-                // the table of this tile (loaded a tile ago), the loads of the next one, the offsets
-                // of the one after: nothing here waits for memory
-                if (pt * 16 < p.tab_bytes)
-                    *reinterpret_cast<uint4 *>(smem_raw + tab_off + (size_t)buf * p.tab_bytes + pt * 16) = tabv;
-                if (pt == 0) ctr[buf] = 0;
-                if (n_c + 1 < n_tiles) {
-                    const unsigned char *nrec = p.sched + off0;
-                    if (pt * 16 < p.tab_bytes) tabv = load_u4(nrec + pt * 16);
-                    for (uint64_t o = (uint64_t)pt * 128u; o < off1 - off0; o += (uint64_t)kProducerWarps * 32u * 128u)   // the record into L2 ahead of its walk
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(nrec + o));
-                }
-                if (n_c + 2 < n_tiles) {
-                    const int64_t t2 = c + (n_c + 2) * p.cpg;
-                    off0 = load_u64(p.sched_off + t2);
-                    off1 = load_u64(p.sched_off + t2 + 1);
-                }
-                prefetch_tile(n_c + 2);
-                block_barrier<kThreads>();
-                b_c = 0;
-                ++n_c;
             }
+            // the table of this tile (loaded a tile ago), the loads of the next one, the offsets
+            // of the one after: nothing here waits for memory
+            if (pt * 16 < p.tab_bytes)
+                *reinterpret_cast<uint4 *>(smem_raw + tab_off + (size_t)buf * p.tab_bytes + pt * 16) = tabv;
+            if (pt == 0) ctr[buf] = 0;
+            if (n + 1 < n_tiles) {
+                const unsigned char *nrec = p.sched + off0;
+                if (pt * 16 < p.tab_bytes) tabv = load_u4(nrec + pt * 16);
+                for (uint64_t o = (uint64_t)pt * 128u; o < off1 - off0; o += (uint64_t)kProducerWarps * 32u * 128u)   // the record into L2 ahead of its walk
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(nrec + o));
+            }
+            if (n + 2 < n_tiles) {
+                const int64_t t2 = c + (n + 2) * p.cpg;
+                off0 = load_u64(p.sched_off + t2);
+                off1 = load_u64(p.sched_off + t2 + 1);
+            }
+            prefetch_tile(n + 2);
+            block_barrier<kThreads>();
         };
+
+        if constexpr (!MEAN) {
+            // workers past K alias the group's first row (their sums are computed and never written
+            // out), so the loop below needs no per-worker predicate
+            int64_t roff[GW];
 #pragma unroll
-        for (int s = 0; s < kDepth; ++s) issue(s);
-        while (n_c < n_tiles) {
+            for (int k = 0; k < GW; ++k) roff[k] = g * GW + k < p.K ? (int64_t)k * p.row_stride : 0;
+            float4 wv[kDepth][GW], w0v[kDepth], xv[kDepth];       // four consecutive indices each
+            int64_t n_i = 0, n_c = 0;                             // tile being loaded / stored
+            int b_i = 0, b_c = 0;                                 // batch inside it
+            int64_t j_i = (int64_t)c * T + 4 * pt;                // first index of this thread's next loads
+            int64_t end_i = (int64_t)(c + 1) * T;                 // end of the tile they belong to
+            const int64_t wrap = (int64_t)(p.cpg - 1) * T;        // from the end of a tile to this block's next one
+            auto issue = [&](int slot) {
+                if (n_i < n_tiles) {
+                    const float *q = wbase + j_i;
+                    if (vec_in && end_i <= p.d) {                 // a whole tile of aligned rows: 128-bit loads
 #pragma unroll
-            for (int s = 0; s < kDepth; ++s) {
-                if (n_c < n_tiles) { consume(s); issue(s); }
+                        for (int k = 0; k < GW; ++k) wv[slot][k] = load4_stream(q + roff[k]);
+                        w0v[slot] = load4_keep(p.w_t0 + j_i);
+                        if (LINEAR) xv[slot] = load4_keep(p.xi + j_i);
+                    } else {                                      // the last tile of the model, or unaligned rows
+                        const int64_t left = p.d - j_i;
+                        const int n = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
+                        const bool vec = vec_in && n == 4;
+#pragma unroll
+                        for (int k = 0; k < GW; ++k) wv[slot][k] = load_quad<true>(q + roff[k], vec, n);
+                        w0v[slot] = load_quad<false>(p.w_t0 + j_i, vec, n);
+                        if (LINEAR) xv[slot] = load_quad<false>(p.xi + j_i, vec, n);
+                    }
+                    j_i += kBatch;
+                    if (++b_i == p.nb) { b_i = 0; ++n_i; j_i += wrap; end_i += wrap + T; }
+                }
+            };
+            auto consume = [&](int slot) {
+                const int buf = (int)(n_c & 1);
+                // rows 4*pt .. 4*pt+3 of the batch; row r is stored at r ^ ((r >> 3) & 3), so that the
+                // eight lanes of a store pass hit eight different bank groups (the schedule's entries
+                // hold the swizzled row)
+                const uint32_t r0 = (uint32_t)(b_c * kBatch + 4 * pt);
+                const uint32_t dst0 = smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 16u;
+                const uint32_t sw = (r0 >> 3) & 3u;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float w0 = comp(w0v[slot], q);
+                    const float u0 = comp(wv[slot][0], q) - w0;
+                    const float u1 = comp(wv[slot][1], q) - w0;
+                    const float u2 = comp(wv[slot][2], q) - w0;
+                    const float u3 = comp(wv[slot][3], q) - w0;
+                    nf[0] = fmaf(u0, u0, nf[0]); nf[1] = fmaf(u1, u1, nf[1]);
+                    nf[2] = fmaf(u2, u2, nf[2]); nf[3] = fmaf(u3, u3, nf[3]);
+                    if (LINEAR) {
+                        const float xq = comp(xv[slot], q);
+                        pf[0] = fmaf(xq, u0, pf[0]); pf[1] = fmaf(xq, u1, pf[1]);
+                        pf[2] = fmaf(xq, u2, pf[2]); pf[3] = fmaf(xq, u3, pf[3]);
+                    }
+                    store_row(dst0 + (((uint32_t)q ^ sw) << 4), u0, u1, u2, u3);
+                }
+                if (++b_c == p.nb) {
+                    end_of_tile(n_c);
+                    b_c = 0;
+                    ++n_c;
+                }
+            };
+#pragma unroll
+            for (int s = 0; s < kDepth; ++s) issue(s);
+            while (n_c < n_tiles) {
+#pragma unroll
+                for (int s = 0; s < kDepth; ++s) {
+                    if (n_c < n_tiles) { consume(s); issue(s); }
+                }
+            }
+        } else {
+            // Rows are taken four at a time (a chunk): the workers 4*ch .. 4*ch+3, fewer in the last
+            // chunk.  A warp has the loads of one chunk in flight: the next chunk (of this quad, of the
+            // next batch, of the next tile) is asked for as soon as the registers are free.  One running
+            // sum per index: more would not fit the 72 registers that 28 warps leave a thread.
+            const int n_chunks = (p.K + GW - 1) / GW;
+            float4 wv[GW], w0v, xv, acc;                          // acc: the drifts of the quad's indices, summed over the workers so far
+            w0v = make_float4(0.f, 0.f, 0.f, 0.f);
+            xv = make_float4(0.f, 0.f, 0.f, 0.f);
+            acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            auto issue = [&](int64_t j, bool whole, int ch) {
+                const int nv = p.K - ch * GW;                     // rows of this chunk (4 or more: all four)
+                const float *q = p.w + (size_t)(ch * GW) * (size_t)p.row_stride + j;
+                if (whole) {
+#pragma unroll
+                    for (int k = 0; k < GW; ++k)
+                        if (k < nv) wv[k] = load4_stream(q + (int64_t)k * p.row_stride);
+                    if (ch == 0) {
+                        if (!p.base_zero) w0v = load4_keep(p.w_t0 + j);
+                        if (LINEAR) xv = load4_keep(p.xi + j);
+                    }
+                } else {                                          // the last tile of the model, or unaligned rows
+                    const int64_t left = p.d - j;
+                    const int nn = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
+                    const bool vec = vec_in && nn == 4;
+#pragma unroll
+                    for (int k = 0; k < GW; ++k)
+                        if (k < nv) wv[k] = load_quad<true>(q + (int64_t)k * p.row_stride, vec, nn);
+                    if (ch == 0) {
+                        if (!p.base_zero) w0v = load_quad<false>(p.w_t0 + j, vec, nn);
+                        if (LINEAR) xv = load_quad<false>(p.xi + j, vec, nn);
+                    }
+                }
+            };
+            auto consume = [&](int buf, int b, int ch) {
+                const int nv = p.K - ch * GW;
+#pragma unroll
+                for (int k = 0; k < GW; ++k) {
+                    if (k < nv) {
+                        const float ux = wv[k].x - w0v.x, uy = wv[k].y - w0v.y, uz = wv[k].z - w0v.z, uw = wv[k].w - w0v.w;
+                        nf[0] = fmaf(ux, ux, nf[0]); nf[0] = fmaf(uy, uy, nf[0]);
+                        nf[0] = fmaf(uz, uz, nf[0]); nf[0] = fmaf(uw, uw, nf[0]);
+                        acc.x += ux; acc.y += uy; acc.z += uz; acc.w += uw;
+                    }
+                }
+                if (ch + 1 == n_chunks) {                         // the quad is complete: rows 4*pt .. 4*pt+3 of the batch
+                    const uint32_t r0 = (uint32_t)(b * kBatch + 4 * pt);
+                    const uint32_t dst0 = smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 16u;
+                    const uint32_t sw = (r0 >> 3) & 3u;           // row r is stored at r ^ ((r >> 3) & 3)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float sq = comp(acc, q);
+                        if (LINEAR) pf[0] = fmaf(comp(xv, q), sq, pf[0]);
+                        store_row(dst0 + (((uint32_t)q ^ sw) << 4), sq, 0.f, 0.f, 0.f);
+                    }
+                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            };
+            const int64_t tile_stride = (int64_t)p.cpg * T;
+            int64_t tile0 = (int64_t)c * T;                       // first index of the tile being stored
+            issue(tile0 + 4 * pt, vec_in && tile0 + T <= p.d, 0);
+            for (int64_t n = 0; n < n_tiles; ++n, tile0 += tile_stride) {
+                const int buf = (int)(n & 1);
+                const bool whole = vec_in && tile0 + T <= p.d;
+                const bool next_whole = vec_in && tile0 + tile_stride + T <= p.d;
+                for (int b = 0; b < p.nb; ++b) {
+                    const int64_t j = tile0 + (int64_t)b * kBatch + 4 * pt;
+                    for (int ch = 0; ch < n_chunks; ++ch) {
+                        consume(buf, b, ch);
+                        if (ch + 1 < n_chunks) issue(j, whole, ch + 1);
+                        else if (b + 1 < p.nb) issue(j + kBatch, whole, 0);
+                        else if (n + 1 < n_tiles) issue(tile0 + tile_stride + 4 * pt, next_whole, 0);
+                    }
+                }
+                end_of_tile(n);
             }
         }
     } else {
@@ -377,9 +485,10 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
         for (int t = tid; t < lm * GW; t += kThreads) out[t] = bins[t];
     }
     // ---- block partial of (||u||^2, <xi,u>) per worker: the producer warps' sums, in warp order ----
-    if (tid < GW * 2) {
+    // (MEAN: one pair per block, the sum over all workers)
+    if (tid < (MEAN ? 2 : GW * 2) && !(MEAN && p.sketch_only)) {
         double t = 0.0;
-        for (int q = 0; q < kProducerWarps; ++q) t += sums[q * GW * 2 + tid];
+        for (int q = 0; q < kProducerWarps; ++q) t += sums[q * (MEAN ? 2 : GW * 2) + tid];
         p.part_np[(size_t)blockIdx.x * GW * 2 + tid] = t;
     }
 }
@@ -429,40 +538,88 @@ __global__ void k_finalize_gather(const ListParams p, int blocks, uint32_t flags
     }
 }
 
-template <int PW, int WW>
+// Averaged state: mean_state[e] = (sum over the blocks, and over the four columns of a cell, of the
+// partials) / divisor, in fp64 and in a fixed order (column after column, block after block, eight
+// loads in flight).  The two scalars are summed from np_src[b * np_pitch + e], b < np_blocks - this
+// kernel's own partials, or those of the pass that averaged the drifts - and divided by K.
+__global__ void k_finalize_gather_mean(const ListParams p, int blocks, uint32_t flags, const double *__restrict__ np_src,
+                                       int np_blocks, int np_pitch, double cell_div, float *__restrict__ mean_state)
+{
+    const int lm = p.l * p.m;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && warp < 2) {          // the scalars: lanes stride the partials, fixed shuffle tree
+        const int e = warp;
+        const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0 : ((flags & FDA_STATE_LINEAR) != 0 && p.have_xi);
+        double acc = 0.0;
+        if (on)
+            for (int b = lane; b < np_blocks; b += 32) acc += np_src[(size_t)b * np_pitch + e];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) mean_state[e] = (float)(acc / (double)p.K);
+    }
+    const int cell = blockIdx.x * blockDim.x + threadIdx.x;
+    if (cell >= lm) return;
+    double acc = 0.0;
+    if (flags & FDA_STATE_SKETCH) {
+        for (int k = 0; k < GW; ++k) {
+            const float *src = p.part_sk + (size_t)cell * GW + k;
+            double a = 0.0;
+            int b = 0;
+            for (; b + 8 <= blocks; b += 8) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(b + u) * lm * GW];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) a += (double)v[u];
+            }
+            for (; b < blocks; ++b) a += (double)src[(size_t)b * lm * GW];
+            acc += a;
+        }
+    }
+    mean_state[2 + cell] = (float)(acc / cell_div);
+}
+
+template <bool MEAN, int PW, int WW>
 cudaError_t launch_lists(ListParams &p, int blocks, size_t smem, int smem_optin, cudaStream_t s)
 {
     if (p.T % (PW * 128) != 0 || PW * 32 * 16 < p.tab_bytes) return cudaErrorNotSupported;
     p.nb = p.T / (PW * 128);
-    auto kern = p.have_xi ? k_local_state_gather<true, PW, WW> : k_local_state_gather<false, PW, WW>;
+    auto kern = p.have_xi ? k_local_state_gather<true, MEAN, PW, WW> : k_local_state_gather<false, MEAN, PW, WW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
     if (e != cudaSuccess) return e;
     kern<<<blocks, (PW + WW) * 32, smem, s>>>(p);
     return cudaGetLastError();
 }
 
-}  // namespace
+enum ListMode { kPerWorker, kMeanFused, kMeanOfVector };
 
-// Returns cudaErrorNotSupported when the request does not fit this path (the caller then uses
-// the other kernels); any other value is the result of the launches.
-cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
-                                          int64_t d, const float *w_t0, const float *xi,
-                                          uint32_t flags, float *states, cudaStream_t s)
+// kPerWorker: states[K][.] of the K rows of w.  kMeanFused: the averaged state of the K rows in one
+// pass.  kMeanOfVector: w is one row that holds the average drift already (w_t0 unused); the cells
+// of the averaged state come from it, the two scalars from np_blocks partial pairs that the
+// averaging pass left at the start of ctx->part_np, and K only divides those.
+cudaError_t launch_list_kernel(fda_ctx *ctx, ListMode mode, const float *w, int64_t row_stride, int K, int64_t d,
+                               const float *w_t0, const float *xi, bool have_xi, uint32_t flags, float *out,
+                               int np_blocks, cudaStream_t s)
 {
     if (!(flags & FDA_STATE_SKETCH) || ctx->l == 0 || !ctx->sched) return cudaErrorNotSupported;
-    const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
+    const float *xi_used = (mode != kMeanOfVector && (flags & FDA_STATE_LINEAR)) ? xi : nullptr;
+    const bool mean = mode != kPerWorker;
+    const int rows = mode == kMeanOfVector ? 1 : K;
 
     ListParams p{};
     p.w = w; p.w_t0 = w_t0; p.xi = xi_used; p.row_stride = row_stride;
-    p.K = K; p.d = d; p.have_xi = xi_used != nullptr;
-    p.vec = ((((uintptr_t)w | (uintptr_t)w_t0 | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) && (row_stride % 4 == 0);
+    p.K = rows; p.d = d; p.have_xi = xi_used != nullptr;
+    p.base_zero = mode == kMeanOfVector;
+    p.sketch_only = mode == kMeanOfVector;
+    p.vec = ((((uintptr_t)w | (uintptr_t)(p.base_zero ? w : w_t0) | (uintptr_t)(xi_used ? xi_used : w)) & 15u) == 0) &&
+            (row_stride % 4 == 0);
     p.l = ctx->l; p.m = ctx->m;
     p.T = ctx->sched_T;
     p.sched = ctx->sched; p.sched_off = ctx->sched_off;
     p.part_sk = ctx->part_sk; p.part_np = ctx->part_np;
     p.tiles = (d + p.T - 1) / p.T;
     p.tab_bytes = fda_list_table_bytes(ctx->sched_ni_max);
-    p.groups = (K + GW - 1) / GW;
+    p.groups = mean ? 1 : (K + GW - 1) / GW;
     if (p.groups > ctx->n_sm) return cudaErrorNotSupported;
     int64_t cpg = ctx->n_sm / p.groups;
     if (cpg > p.tiles) cpg = p.tiles;
@@ -476,16 +633,62 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     const size_t smem = fda_list_smem_bytes(p.l, p.m, p.T, ctx->sched_ni_max);
     if (smem > (size_t)ctx->smem_optin) return cudaErrorNotSupported;
 
+    cudaError_t e = cudaErrorNotSupported;
+    if (mean) {
+        // The averaged state walks l updates per index however many rows are loaded for it: 12
+        // producer warps when the K rows are read here and the tile divides into their batches of
+        // 1536 indices (5 x 250, K = 8, d = 198M: 2.15 ms against 2.82 ms with 8), else 8.
+        if (mode == kMeanFused) e = launch_lists<true, 12, 16>(p, blocks, smem, ctx->smem_optin, s);
+        if (e == cudaErrorNotSupported) e = launch_lists<true, 8, 20>(p, blocks, smem, ctx->smem_optin, s);
+        if (e != cudaSuccess) return e;
+        const int fblocks = ((ctx->lm > 64 ? ctx->lm : 64) + 127) / 128;      // at least two warps for the scalars
+        p.K = K;
+        p.have_xi = have_xi;
+        if (mode == kMeanFused)
+            k_finalize_gather_mean<<<fblocks, 128, 0, s>>>(p, blocks, flags, ctx->part_np, blocks, GW * 2, (double)K, out);
+        else
+            k_finalize_gather_mean<<<fblocks, 128, 0, s>>>(p, blocks, flags, ctx->part_np, np_blocks, 2, 1.0, out);
+        return cudaGetLastError();
+    }
     // 8 producer + 20 walker warps, or 4 + 24 when a loaded index pays for more walking.  Measured:
     // 7 x 500, K = 60, d = 20M: 3.34 ms with 4 + 24 against 3.71 ms with 8 + 20; 5 x 250, K = 8,
     // d = 198M: 3.49 against 2.49 ms; 5 x 250, K = 30, d = 7M: 0.535 against 0.387 ms.
-    cudaError_t e;
-    if (ctx->l >= 7) e = launch_lists<4, 24>(p, blocks, smem, ctx->smem_optin, s);
-    else e = launch_lists<8, 20>(p, blocks, smem, ctx->smem_optin, s);
+    if (ctx->l >= 7) e = launch_lists<false, 4, 24>(p, blocks, smem, ctx->smem_optin, s);
+    else e = launch_lists<false, 8, 20>(p, blocks, smem, ctx->smem_optin, s);
     if (e != cudaSuccess) return e;
     const int64_t total = (int64_t)p.groups * (2 + ctx->lm) * GW * 4;
     int fb = (int)((total + 255) / 256);
     if (fb > ctx->n_sm * 8) fb = ctx->n_sm * 8;
-    k_finalize_gather<<<fb, 256, 0, s>>>(p, blocks, flags, states);
+    k_finalize_gather<<<fb, 256, 0, s>>>(p, blocks, flags, out);
     return cudaGetLastError();
+}
+
+}  // namespace
+
+// Returns cudaErrorNotSupported when the request does not fit this path (the caller then uses
+// the other kernels); any other value is the result of the launches.
+cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                          int64_t d, const float *w_t0, const float *xi,
+                                          uint32_t flags, float *states, cudaStream_t s)
+{
+    return launch_list_kernel(ctx, kPerWorker, w, row_stride, K, d, w_t0, xi, false, flags, states, 0, s);
+}
+
+// The averaged state S-bar of fda_mean_state on the same kernel, in one pass over the K rows; same
+// return convention.
+cudaError_t fda_launch_mean_state_gather(fda_ctx *ctx, const float *w, int64_t row_stride, int K,
+                                         int64_t d, const float *w_t0, const float *xi,
+                                         uint32_t flags, float *mean_state, cudaStream_t s)
+{
+    const bool have_xi = (flags & FDA_STATE_LINEAR) && xi;
+    return launch_list_kernel(ctx, kMeanFused, w, row_stride, K, d, w_t0, xi, have_xi, flags, mean_state, 0, s);
+}
+
+// The cells of S-bar from the vector of averaged drifts (d floats, 16-byte aligned), the scalars
+// from the np_blocks partial pairs at the start of ctx->part_np; same return convention.
+cudaError_t fda_launch_mean_sketch_gather(fda_ctx *ctx, const float *mean_drift, int K, int64_t d, bool have_xi,
+                                          uint32_t flags, int np_blocks, float *mean_state, cudaStream_t s)
+{
+    return launch_list_kernel(ctx, kMeanOfVector, mean_drift, (d + 3) / 4 * 4, K, d, nullptr, nullptr, have_xi, flags,
+                              mean_state, np_blocks, s);
 }

@@ -342,9 +342,21 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
 {
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
-    if (sketch) {                // first use: the 16-bit hash table
-        const cudaError_t e = fda_ensure_table(ctx, s);
-        if (e != cudaSuccess) return e;
+    // With a list schedule in the context the cells can come from the list kernel.  In one pass over
+    // the K rows when there are few of them and the vector is long: 2.15 against 2.58 ms at 5 x 250,
+    // K = 8, d = 198M, but no gain at d = 7M, where the averaged drifts and the 16-bit table of the
+    // two-pass route stay in L2.  From the averaged drifts that phase 1 leaves in memory when the
+    // sketch is too large for the lane-private bins of k_sketch_vector_rows: 1.02 against 1.42 ms at
+    // 7 x 500, K = 60, d = 20M (at 5 x 250 that kernel is the faster one: 0.22 against 0.25 ms at
+    // K = 30, d = 7M).
+    const bool lists = sketch && ctx->sched != nullptr;
+    const int64_t tiles = lists ? (d + ctx->sched_T - 1) / ctx->sched_T : 0;
+    if (lists && K <= 2 * ctx->l && tiles >= 8 * (int64_t)ctx->n_sm) {
+        const cudaError_t e = fda_launch_mean_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, mean_state, s);
+        if (e != cudaErrorNotSupported) {
+            if (e == cudaSuccess) ctx->last_ls_kernel = "k_local_state_gather(mean)";
+            return e;
+        }
     }
     if (!ctx->mean_model) {      // first use: d_max floats of scratch for the average drift
         cudaError_t e = cudaMalloc(&ctx->mean_model, sizeof(float) * (size_t)((ctx->d_max + 3) / 4 * 4));
@@ -369,8 +381,18 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
     if (e != cudaSuccess) return e;
 
     // phase 2: sketch of u-bar
+    if (lists && ctx->columns != 32) {
+        e = fda_launch_mean_sketch_gather(ctx, ctx->mean_model, K, d, linear, flags, (int)nblk, mean_state, s);
+        if (e != cudaErrorNotSupported) {
+            if (e == cudaSuccess) ctx->last_ls_kernel = "k_mean_model + k_local_state_gather(mean)";
+            return e;
+        }
+    }
+    ctx->last_ls_kernel = sketch ? "k_mean_model + k_sketch_vector" : "k_mean_model";
     int sk_blocks = 0;
     if (sketch) {
+        e = fda_ensure_table(ctx, s);        // first use: the 16-bit hash table
+        if (e != cudaSuccess) return e;
         SketchVecParams p{};
         p.v = ctx->mean_model; p.d = d; p.tab = ctx->tab; p.tab_stride = ctx->tab_stride;
         p.l = ctx->l; p.m = ctx->m; p.lm = ctx->lm; p.cshift = ilog2(ctx->columns); p.part_sk = ctx->part_sk;

@@ -11,7 +11,7 @@ import numpy as np
 import pytest
 
 import fda_synth as S
-from fda_testlib import check_states
+from fda_testlib import check_mean_state, check_states
 
 pytestmark = pytest.mark.gpu
 
@@ -191,6 +191,7 @@ def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
         assert ctx.fda_debug_last_kernel() == GATHER and ctx.fda_context_info()["table_bytes"] == 0
         mean = torch.empty((ctx.state_len,), device="cuda")
         ctx.fda_mean_state(w, w0, None, 1 | 4, mean)                         # first use builds the 16-bit table
+        assert ctx.fda_debug_last_kernel() == "k_mean_model + k_sketch_vector"
         after = ctx.fda_context_info()
         assert after["table_bytes"] >= 2 * l * d and after["other_lazy_bytes"] >= 4 * d
         torch.cuda.synchronize()
@@ -209,6 +210,35 @@ def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
             n = ref[:, :1]
             scale = np.maximum(np.abs(ref), np.sqrt(n / m))
             assert float(np.max(np.abs(got - ref) / scale)) <= 2e-5        # two fp32 paths, each within 1e-5 of the oracle
+
+
+def test_averaged_state_routes(env):
+    """Which kernels serve fda_mean_state, and what scratch they make the context allocate: a long
+    vector with few workers goes through the list kernel in one pass (nothing allocated); a sketch
+    too large for lane-private bins gets its cells from the list kernel run on the averaged drifts
+    (d floats, no hash table).  Both against the average of the oracle's per-worker states."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(27)
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    for K, d, l, m, want, lazy in [
+        (4, 6144 * 8 * n_sm + 13, 5, 250, "k_local_state_gather(mean)", False),
+        (20, 300_007, 7, 500, "k_mean_model + k_local_state_gather(mean)", True),
+    ]:
+        coeffs = rand_coeffs(rng, l)
+        w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+        wbuf = w_t0 + rng.normal(2e-4, 1e-3, size=(K, d)).astype(np.float32)
+        ora = oracle.local_state(wbuf, w_t0, None, coeffs, l, m, threads=8)
+        _, _, ubar_sq = oracle.variance(wbuf, w_t0)
+        with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+            assert ctx.fda_context_info()["list_kernel"] == 1
+            mean = torch.full((ctx.state_len,), float("nan"), device="cuda")
+            ctx.fda_mean_state(torch.from_numpy(wbuf).cuda(), torch.from_numpy(w_t0).cuda(), None, 1 | 4, mean)
+            torch.cuda.synchronize()
+            assert ctx.fda_debug_last_kernel() == want
+            after = ctx.fda_context_info()
+            assert after["table_bytes"] == 0
+            assert (4 * d <= after["other_lazy_bytes"] < 5 * d) if lazy else after["other_lazy_bytes"] == 0
+            check_mean_state(mean.cpu().numpy(), ora, ubar_sq, l, m, d, K)
 
 
 def test_more_worker_groups_than_the_scratch_holds_are_refused(env):
