@@ -57,6 +57,8 @@ struct ListParams {
     float *part_sk;                  // [block][cell][GW]
     double *part_np;                 // [block][GW][2]
     int base_zero;                   // averaged state only: the rows are drifts already (no w_t0 to subtract)
+    int depth;                       // averaged state only: quads a producer thread keeps in flight in its
+                                     // shared-memory landing zone (1..8)
     int sketch_only;                 // averaged state only: leave part_np alone
 };
 
@@ -136,6 +138,47 @@ __device__ __forceinline__ void gather_hi(uint32_t w, uint32_t base, unsigned lo
     gather_row((w >> 12) & 0x1fff0u, (w & 0x80000000u) ^ 0x3f800000u, base, a01, a23);
 }
 
+// 16 bytes from global memory straight into shared memory (no register in between), in groups
+// that the issuing thread waits for by age.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const float *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// four bytes (on == false: four zero bytes, src is not read)
+__device__ __forceinline__ void cp_async4(uint32_t dst, const float *src, bool on)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(on ? 4 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// returns when at most n (0..7) of the thread's groups are still in flight
+__device__ __forceinline__ void cp_async_wait_upto(int n)
+{
+    switch (n) {
+        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+    }
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// One entry of a single-column tile (the averaged state): a 32-bit load, the sign flips the top bit.
+__device__ __forceinline__ void gather1(uint32_t e, uint32_t base, float &a)
+{
+    float u;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(u) : "r"(base + ((e & 0x1fffu) << 2)));
+    a += __uint_as_float(__float_as_uint(u) ^ ((e & 0x8000u) << 16));
+}
+
 // Shared-memory plan (bytes from the start of dynamic shared memory):
 //   [0, 8)    item counters of the two tile buffers
 //   [64, 1088) sums[producer warp][worker][2] (fp64): ||u||^2 and <xi,u> over the tiles so far
@@ -145,9 +188,9 @@ __device__ __forceinline__ void gather_hi(uint32_t w, uint32_t base, unsigned lo
 // PW producer warps and WW walker warps: the split that is fastest depends on how much walking a
 // loaded index pays for (l updates per worker).
 // MEAN (the averaged state of fda_mean_state; by linearity, Section 3.1 (a), the sketch of the
-// mean drift): one block group serves all K workers, the first column of a row of the tile holds
-// the sum of all workers' drifts and the other three are zero, so the walk costs l updates per
-// index instead of K*l; the sums are divided by K at the end.
+// mean drift): one block group serves all K workers, a row of the tile is one float, the sum of all
+// workers' drifts of the index, and a cell of the bins one float, so the walk costs l 4-byte reads
+// per index instead of K*l; the sums are divided by K at the end.
 template <bool LINEAR, bool MEAN, int PW, int WW>
 __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const ListParams p)
 {
@@ -166,14 +209,15 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
     double *sums = reinterpret_cast<double *>(smem_raw + 64);
     const uint32_t tab_off = kListSmemHead;
     const uint32_t bins_off = tab_off + 2u * (uint32_t)p.tab_bytes;
-    const uint32_t ut_off = bins_off + (uint32_t)lm * 16u;
-    const uint32_t ut_bytes = (uint32_t)(T + kListPadRows) * 16u;
+    constexpr int COLS = MEAN ? 1 : GW;                       // floats per row of the drift tile and per cell of the bins
+    const uint32_t ut_off = bins_off + (uint32_t)lm * 16u;    // (MEAN uses a quarter of the bins and of each tile buffer)
+    const uint32_t ut_bytes = (uint32_t)(T + kListPadRows) * 4u * COLS;
     float *bins = reinterpret_cast<float *>(smem_raw + bins_off);
 
-    for (int t = tid; t < lm * GW; t += kThreads) bins[t] = 0.f;
-    for (int t = tid; t < 2 * kListPadRows * GW; t += kThreads) {
-        const int b = t / (kListPadRows * GW), r = t % (kListPadRows * GW);
-        reinterpret_cast<float *>(smem_raw + ut_off + (size_t)b * ut_bytes)[T * GW + r] = 0.f;
+    for (int t = tid; t < lm * COLS; t += kThreads) bins[t] = 0.f;
+    for (int t = tid; t < 2 * kListPadRows * COLS; t += kThreads) {
+        const int b = t / (kListPadRows * COLS), r = t % (kListPadRows * COLS);
+        reinterpret_cast<float *>(smem_raw + ut_off + (size_t)b * ut_bytes)[T * COLS + r] = 0.f;
     }
     if (tid < 2) ctr[tid] = 0;
     if (tid < kMaxProducerWarps * GW * 2) sums[tid] = 0.0;
@@ -340,81 +384,86 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
                 }
             }
         } else {
-            // Rows are taken four at a time (a chunk): the workers 4*ch .. 4*ch+3, fewer in the last
-            // chunk.  A warp has the loads of one chunk in flight: the next chunk (of this quad, of the
-            // next batch, of the next tile) is asked for as soon as the registers are free.  One running
-            // sum per index: more would not fit the 72 registers that 28 warps leave a thread.
-            const int n_chunks = (p.K + GW - 1) / GW;
-            float4 wv[GW], w0v, xv, acc;                          // acc: the drifts of the quad's indices, summed over the workers so far
-            w0v = make_float4(0.f, 0.f, 0.f, 0.f);
-            xv = make_float4(0.f, 0.f, 0.f, 0.f);
-            acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            auto issue = [&](int64_t j, bool whole, int ch) {
-                const int nv = p.K - ch * GW;                     // rows of this chunk (4 or more: all four)
-                const float *q = p.w + (size_t)(ch * GW) * (size_t)p.row_stride + j;
-                if (whole) {
+            // The single-column tile leaves most of the shared memory free, so the loads land there
+            // instead of in registers: the rows of a quad of indices (the K workers, w_t0, xi) are
+            // copied asynchronously, `depth` quads ahead per thread, and the thread that asked for
+            // them reads them back when their group has landed.  The bytes in flight then depend
+            // neither on registers nor on the number of producer warps (with the loads in registers,
+            // four rows at a time, the same pass took 2.07 instead of 1.73 ms at K = 8, d = 198M).
+            // Slot s, row r of thread pt: lz + ((s * R + r) * threads + pt) * 16.  Elements past d and
+            // the rows of a model that is not 16-byte aligned are copied four bytes at a time, with
+            // zeros for what lies past the end.
+            const int D = p.depth;
+            const int R = p.K + (p.base_zero ? 0 : 1) + (LINEAR ? 1 : 0);
+            constexpr uint32_t kRowPitch = (uint32_t)kProducerWarps * 32u * 16u;
+            const uint32_t lz = smem_base + ut_off + 2u * ut_bytes + (uint32_t)pt * 16u;
+            const int64_t quads = n_tiles * p.nb;                 // this thread's quads
+            int64_t s_i = 0;                                      // next quad to ask for
+            int b_i = 0;
+            int64_t j_i = (int64_t)c * T + 4 * pt;
+            const int64_t wrap = (int64_t)(p.cpg - 1) * T;        // from the end of a tile to this block's next one
+            // the slow copy: what lies past d becomes zero
+            auto copy_ragged = [&](uint32_t dst, const float *row, int64_t j) {
+                const int64_t left = p.d - j;
 #pragma unroll
-                    for (int k = 0; k < GW; ++k)
-                        if (k < nv) wv[k] = load4_stream(q + (int64_t)k * p.row_stride);
-                    if (ch == 0) {
-                        if (!p.base_zero) w0v = load4_keep(p.w_t0 + j);
-                        if (LINEAR) xv = load4_keep(p.xi + j);
-                    }
-                } else {                                          // the last tile of the model, or unaligned rows
-                    const int64_t left = p.d - j;
-                    const int nn = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
-                    const bool vec = vec_in && nn == 4;
-#pragma unroll
-                    for (int k = 0; k < GW; ++k)
-                        if (k < nv) wv[k] = load_quad<true>(q + (int64_t)k * p.row_stride, vec, nn);
-                    if (ch == 0) {
-                        if (!p.base_zero) w0v = load_quad<false>(p.w_t0 + j, vec, nn);
-                        if (LINEAR) xv = load_quad<false>(p.xi + j, vec, nn);
-                    }
-                }
+                for (int e = 0; e < 4; ++e) cp_async4(dst + 4u * e, e < left ? row + j + e : row, e < left);
             };
-            auto consume = [&](int buf, int b, int ch) {
-                const int nv = p.K - ch * GW;
-#pragma unroll
-                for (int k = 0; k < GW; ++k) {
-                    if (k < nv) {
-                        const float ux = wv[k].x - w0v.x, uy = wv[k].y - w0v.y, uz = wv[k].z - w0v.z, uw = wv[k].w - w0v.w;
+            auto issue_lz = [&](int slot) {
+                if (s_i < quads) {
+                    const uint32_t dst = lz + (uint32_t)(slot * R) * kRowPitch;
+                    if (vec_in && j_i + 4 <= p.d) {
+                        const float *q = p.w + j_i;
+                        for (int k = 0; k < p.K; ++k) cp_async16(dst + (uint32_t)k * kRowPitch, q + (int64_t)k * p.row_stride);
+                        int r = p.K;
+                        if (!p.base_zero) { cp_async16(dst + (uint32_t)r * kRowPitch, p.w_t0 + j_i); ++r; }
+                        if (LINEAR) cp_async16(dst + (uint32_t)r * kRowPitch, p.xi + j_i);
+                    } else {
+                        for (int k = 0; k < p.K; ++k) copy_ragged(dst + (uint32_t)k * kRowPitch, p.w + (int64_t)k * p.row_stride, j_i);
+                        int r = p.K;
+                        if (!p.base_zero) { copy_ragged(dst + (uint32_t)r * kRowPitch, p.w_t0, j_i); ++r; }
+                        if (LINEAR) copy_ragged(dst + (uint32_t)r * kRowPitch, p.xi, j_i);
+                    }
+                    ++s_i;
+                    j_i += kBatch;
+                    if (++b_i == p.nb) { b_i = 0; j_i += wrap; }
+                }
+                cp_async_commit();                                 // (an empty group past the end keeps the count)
+            };
+            for (int s = 0; s < D; ++s) issue_lz(s);
+            int slot = 0;
+            for (int64_t n = 0; n < n_tiles; ++n) {
+                const int buf = (int)(n & 1);
+                for (int b = 0; b < p.nb; ++b) {
+                    cp_async_wait_upto(D - 1);                     // the oldest group has landed
+                    const uint32_t src = lz + (uint32_t)(slot * R) * kRowPitch;
+                    int r = p.K;
+                    float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f), a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (!p.base_zero) { w0 = lds128(src + (uint32_t)r * kRowPitch); ++r; }
+#pragma unroll 4
+                    for (int k = 0; k < p.K; ++k) {
+                        const float4 v = lds128(src + (uint32_t)k * kRowPitch);
+                        const float ux = v.x - w0.x, uy = v.y - w0.y, uz = v.z - w0.z, uw = v.w - w0.w;
                         nf[0] = fmaf(ux, ux, nf[0]); nf[0] = fmaf(uy, uy, nf[0]);
                         nf[0] = fmaf(uz, uz, nf[0]); nf[0] = fmaf(uw, uw, nf[0]);
-                        acc.x += ux; acc.y += uy; acc.z += uz; acc.w += uw;
+                        a.x += ux; a.y += uy; a.z += uz; a.w += uw;
                     }
-                }
-                if (ch + 1 == n_chunks) {                         // the quad is complete: rows 4*pt .. 4*pt+3 of the batch
+                    if (LINEAR) {
+                        const float4 x = lds128(src + (uint32_t)r * kRowPitch);
+                        pf[0] = fmaf(x.x, a.x, pf[0]); pf[0] = fmaf(x.y, a.y, pf[0]);
+                        pf[0] = fmaf(x.z, a.z, pf[0]); pf[0] = fmaf(x.w, a.w, pf[0]);
+                    }
+                    // rows 4*pt .. 4*pt+3 of the batch; row r is stored at r ^ ((r >> 3) & 3): one 16-byte
+                    // store of the quad, its floats permuted
                     const uint32_t r0 = (uint32_t)(b * kBatch + 4 * pt);
-                    const uint32_t dst0 = smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 16u;
-                    const uint32_t sw = (r0 >> 3) & 3u;           // row r is stored at r ^ ((r >> 3) & 3)
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float sq = comp(acc, q);
-                        if (LINEAR) pf[0] = fmaf(comp(xv, q), sq, pf[0]);
-                        store_row(dst0 + (((uint32_t)q ^ sw) << 4), sq, 0.f, 0.f, 0.f);
-                    }
-                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            };
-            const int64_t tile_stride = (int64_t)p.cpg * T;
-            int64_t tile0 = (int64_t)c * T;                       // first index of the tile being stored
-            issue(tile0 + 4 * pt, vec_in && tile0 + T <= p.d, 0);
-            for (int64_t n = 0; n < n_tiles; ++n, tile0 += tile_stride) {
-                const int buf = (int)(n & 1);
-                const bool whole = vec_in && tile0 + T <= p.d;
-                const bool next_whole = vec_in && tile0 + tile_stride + T <= p.d;
-                for (int b = 0; b < p.nb; ++b) {
-                    const int64_t j = tile0 + (int64_t)b * kBatch + 4 * pt;
-                    for (int ch = 0; ch < n_chunks; ++ch) {
-                        consume(buf, b, ch);
-                        if (ch + 1 < n_chunks) issue(j, whole, ch + 1);
-                        else if (b + 1 < p.nb) issue(j + kBatch, whole, 0);
-                        else if (n + 1 < n_tiles) issue(tile0 + tile_stride + 4 * pt, next_whole, 0);
-                    }
+                    const int sw = (int)((r0 >> 3) & 3u);
+                    store_row(smem_base + ut_off + (uint32_t)buf * ut_bytes + r0 * 4u,
+                              comp(a, 0 ^ sw), comp(a, 1 ^ sw), comp(a, 2 ^ sw), comp(a, 3 ^ sw));
+                    issue_lz(slot);                                // the slot is free again
+                    slot = slot + 1 == D ? 0 : slot + 1;
                 }
                 end_of_tile(n);
             }
+            cp_async_wait_upto(0);
         }
     } else {
         // =============================== walkers ===============================
@@ -437,41 +486,72 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
                 const uint32_t cell = cells[(size_t)(d0 >> 16) * kListSlots + lane];
                 const uint2 *ent = reinterpret_cast<const uint2 *>(ent0 + (size_t)chunk0 * 256) + lane;
                 const int nch = (steps + 3) >> 2;
-                unsigned long long a01 = 0ull, a23 = 0ull;
-                // all entry loads of (up to) eight chunks first, then the walk: the entries come
-                // from global memory (L2), one round trip per eight chunks instead of one per chunk
-                for (int c0 = 0; c0 < nch; c0 += kChunksAhead) {
-                    uint2 ch[kChunksAhead];
+                if constexpr (MEAN) {
+                    // one column: a 32-bit load per entry.  The schedule keeps the eight lanes of an
+                    // octet in different banks mod 8; lanes of different octets may still share a bank.
+                    float a = 0.f;
+                    for (int c0 = 0; c0 < nch; c0 += kChunksAhead) {
+                        uint2 ch[kChunksAhead];
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q)
-                        if (c0 + q < nch) ch[q] = __ldg(ent + (size_t)(c0 + q) * kListSlots);
+                        for (int q = 0; q < kChunksAhead; ++q)
+                            if (c0 + q < nch) ch[q] = __ldg(ent + (size_t)(c0 + q) * kListSlots);
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q) {
-                        const int left = steps - 4 * (c0 + q);
-                        if (left >= 4) {
-                            gather_lo(ch[q].x, base, a01, a23);
-                            gather_hi(ch[q].x, base, a01, a23);
-                            gather_lo(ch[q].y, base, a01, a23);
-                            gather_hi(ch[q].y, base, a01, a23);
-                        } else if (left > 0) {
-                            gather_lo(ch[q].x, base, a01, a23);
-                            if (left > 1) gather_hi(ch[q].x, base, a01, a23);
-                            if (left > 2) gather_lo(ch[q].y, base, a01, a23);
+                        for (int q = 0; q < kChunksAhead; ++q) {
+                            const int left = steps - 4 * (c0 + q);
+                            if (left >= 4) {
+                                gather1(ch[q].x & 0xffffu, base, a);
+                                gather1(ch[q].x >> 16, base, a);
+                                gather1(ch[q].y & 0xffffu, base, a);
+                                gather1(ch[q].y >> 16, base, a);
+                            } else if (left > 0) {
+                                gather1(ch[q].x & 0xffffu, base, a);
+                                if (left > 1) gather1(ch[q].x >> 16, base, a);
+                                if (left > 2) gather1(ch[q].y & 0xffffu, base, a);
+                            }
                         }
                     }
-                }
-                float4 acc;
-                asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.x), "=f"(acc.y) : "l"(a01));
-                asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.z), "=f"(acc.w) : "l"(a23));
-                if ((cell & 0x7fffu) < (uint32_t)lm) {
-                    float *b = bins + (cell & 0x7fffu) * GW;
-                    if (cell & 0x8000u) {                           // a cell with several lists
-                        atomicAdd(b + 0, acc.x); atomicAdd(b + 1, acc.y);
-                        atomicAdd(b + 2, acc.z); atomicAdd(b + 3, acc.w);
-                    } else {
-                        float4 o = *reinterpret_cast<float4 *>(b);
-                        o.x += acc.x; o.y += acc.y; o.z += acc.z; o.w += acc.w;
-                        *reinterpret_cast<float4 *>(b) = o;
+                    if ((cell & 0x7fffu) < (uint32_t)lm) {
+                        float *b = bins + (cell & 0x7fffu);
+                        if (cell & 0x8000u) atomicAdd(b, a);            // a cell with several lists
+                        else *b += a;
+                    }
+                } else {
+                    unsigned long long a01 = 0ull, a23 = 0ull;
+                    // all entry loads of (up to) eight chunks first, then the walk: the entries come
+                    // from global memory (L2), one round trip per eight chunks instead of one per chunk
+                    for (int c0 = 0; c0 < nch; c0 += kChunksAhead) {
+                        uint2 ch[kChunksAhead];
+    #pragma unroll
+                        for (int q = 0; q < kChunksAhead; ++q)
+                            if (c0 + q < nch) ch[q] = __ldg(ent + (size_t)(c0 + q) * kListSlots);
+    #pragma unroll
+                        for (int q = 0; q < kChunksAhead; ++q) {
+                            const int left = steps - 4 * (c0 + q);
+                            if (left >= 4) {
+                                gather_lo(ch[q].x, base, a01, a23);
+                                gather_hi(ch[q].x, base, a01, a23);
+                                gather_lo(ch[q].y, base, a01, a23);
+                                gather_hi(ch[q].y, base, a01, a23);
+                            } else if (left > 0) {
+                                gather_lo(ch[q].x, base, a01, a23);
+                                if (left > 1) gather_hi(ch[q].x, base, a01, a23);
+                                if (left > 2) gather_lo(ch[q].y, base, a01, a23);
+                            }
+                        }
+                    }
+                    float4 acc;
+                    asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.x), "=f"(acc.y) : "l"(a01));
+                    asm("mov.b64 {%0,%1}, %2;" : "=f"(acc.z), "=f"(acc.w) : "l"(a23));
+                    if ((cell & 0x7fffu) < (uint32_t)lm) {
+                        float *b = bins + (cell & 0x7fffu) * GW;
+                        if (cell & 0x8000u) {                           // a cell with several lists
+                            atomicAdd(b + 0, acc.x); atomicAdd(b + 1, acc.y);
+                            atomicAdd(b + 2, acc.z); atomicAdd(b + 3, acc.w);
+                        } else {
+                            float4 o = *reinterpret_cast<float4 *>(b);
+                            o.x += acc.x; o.y += acc.y; o.z += acc.z; o.w += acc.w;
+                            *reinterpret_cast<float4 *>(b) = o;
+                        }
                     }
                 }
             }
@@ -481,8 +561,8 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
 
     // ---- flush: bins -> this block's partial sketch ----
     {
-        float *out = p.part_sk + (size_t)blockIdx.x * (size_t)lm * GW;
-        for (int t = tid; t < lm * GW; t += kThreads) out[t] = bins[t];
+        float *out = p.part_sk + (size_t)blockIdx.x * (size_t)lm * COLS;
+        for (int t = tid; t < lm * COLS; t += kThreads) out[t] = bins[t];
     }
     // ---- block partial of (||u||^2, <xi,u>) per worker: the producer warps' sums, in warp order ----
     // (MEAN: one pair per block, the sum over all workers)
@@ -538,9 +618,8 @@ __global__ void k_finalize_gather(const ListParams p, int blocks, uint32_t flags
     }
 }
 
-// Averaged state: mean_state[e] = (sum over the blocks, and over the four columns of a cell, of the
-// partials) / divisor, in fp64 and in a fixed order (column after column, block after block, eight
-// loads in flight).  The two scalars are summed from np_src[b * np_pitch + e], b < np_blocks - this
+// Averaged state: mean_state[e] = (sum over the blocks of the partials) / divisor, in fp64 and in a
+// fixed order (block after block, eight loads in flight).  The two scalars are summed from np_src[b * np_pitch + e], b < np_blocks - this
 // kernel's own partials, or those of the pass that averaged the drifts - and divided by K.
 __global__ void k_finalize_gather_mean(const ListParams p, int blocks, uint32_t flags, const double *__restrict__ np_src,
                                        int np_blocks, int np_pitch, double cell_div, float *__restrict__ mean_state)
@@ -561,20 +640,16 @@ __global__ void k_finalize_gather_mean(const ListParams p, int blocks, uint32_t 
     if (cell >= lm) return;
     double acc = 0.0;
     if (flags & FDA_STATE_SKETCH) {
-        for (int k = 0; k < GW; ++k) {
-            const float *src = p.part_sk + (size_t)cell * GW + k;
-            double a = 0.0;
-            int b = 0;
-            for (; b + 8 <= blocks; b += 8) {
-                float v[8];
+        const float *src = p.part_sk + cell;
+        int b = 0;
+        for (; b + 8 <= blocks; b += 8) {
+            float v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(b + u) * lm * GW];
+            for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(b + u) * lm];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) a += (double)v[u];
-            }
-            for (; b < blocks; ++b) a += (double)src[(size_t)b * lm * GW];
-            acc += a;
+            for (int u = 0; u < 8; ++u) acc += (double)v[u];
         }
+        for (; b < blocks; ++b) acc += (double)src[(size_t)b * lm];
     }
     mean_state[2 + cell] = (float)(acc / cell_div);
 }
@@ -584,6 +659,17 @@ cudaError_t launch_lists(ListParams &p, int blocks, size_t smem, int smem_optin,
 {
     if (p.T % (PW * 128) != 0 || PW * 32 * 16 < p.tab_bytes) return cudaErrorNotSupported;
     p.nb = p.T / (PW * 128);
+    p.depth = 0;
+    if (MEAN) {
+        // what the single-column tile leaves free becomes the producers' landing zone
+        const size_t used = kListSmemHead + 2 * (size_t)p.tab_bytes + (size_t)p.l * p.m * 16 +
+                            2 * (size_t)(p.T + kListPadRows) * 4;
+        const size_t per_quad = (size_t)PW * 32 * 16 * (size_t)(p.K + (p.base_zero ? 0 : 1) + (p.have_xi ? 1 : 0));
+        const size_t depth = (size_t)smem_optin > used ? ((size_t)smem_optin - used) / per_quad : 0;
+        if (depth < 1) return cudaErrorNotSupported;              // too many rows for this route
+        p.depth = (int)(depth < 8 ? depth : 8);
+        smem = used + (size_t)p.depth * per_quad;
+    }
     auto kern = p.have_xi ? k_local_state_gather<true, MEAN, PW, WW> : k_local_state_gather<false, MEAN, PW, WW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
     if (e != cudaSuccess) return e;
@@ -635,11 +721,10 @@ cudaError_t launch_list_kernel(fda_ctx *ctx, ListMode mode, const float *w, int6
 
     cudaError_t e = cudaErrorNotSupported;
     if (mean) {
-        // The averaged state walks l updates per index however many rows are loaded for it: 12
-        // producer warps when the K rows are read here and the tile divides into their batches of
-        // 1536 indices (5 x 250, K = 8, d = 198M: 2.15 ms against 2.82 ms with 8), else 8.
-        if (mode == kMeanFused) e = launch_lists<true, 12, 16>(p, blocks, smem, ctx->smem_optin, s);
-        if (e == cudaErrorNotSupported) e = launch_lists<true, 8, 20>(p, blocks, smem, ctx->smem_optin, s);
+        // 8 producer + 24 walker warps: the single accumulator of the walk and the landing zone of the
+        // loads leave room for 32 warps at 64 registers (K = 8, d = 198M, 5 x 250: 1.67 ms; 1.73 with
+        // 8 + 20, 1.86 with 6 + 26, 2.01 with 12 + 16, 2.12 with 4 + 24).
+        e = launch_lists<true, 8, 24>(p, blocks, smem, ctx->smem_optin, s);
         if (e != cudaSuccess) return e;
         const int fblocks = ((ctx->lm > 64 ? ctx->lm : 64) + 127) / 128;      // at least two warps for the scalars
         p.K = K;
