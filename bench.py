@@ -48,8 +48,8 @@ SMEM_GATHER_UPDATES_PER_CLK_SM = 32.0  # one 4-byte shared-memory read per updat
 # lists summarised under profiles/: profiles/traffic.json names, per workload, the bytes, the
 # summary file and the sha256 of the kernel sources the capture was taken with.  When the sources
 # have changed since, the figure is stale and the bench line says null.
-KERNEL_SOURCES = ("paper_2405_20988_b200/csrc/fda_local_state_gather.cu", "paper_2405_20988_b200/csrc/fda_sched.cu",
-                  "paper_2405_20988_b200/csrc/fda_internal.h")
+KERNEL_SOURCES = ("paper_2405_20988_b200/csrc/fda_local_state_gather.cu", "paper_2405_20988_b200/csrc/fda_list_kernel.cuh",
+                  "paper_2405_20988_b200/csrc/fda_sched.cu", "paper_2405_20988_b200/csrc/fda_internal.h")
 
 
 def kernel_sources_sha256() -> str:

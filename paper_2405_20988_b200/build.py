@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfda.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["fda_api.cu", "fda_hash.cu", "fda_local_state.cu", "fda_local_state_gather.cu", "fda_sched.cu", "fda_local_state_linear.cu", "fda_mean_state.cu", "fda_combine.cu", "fda_average.cu", "fda_noalloc.cu", "fda_probe.cu"]
+SOURCES = ["fda_api.cu", "fda_hash.cu", "fda_local_state.cu", "fda_local_state_gather.cu", "fda_mean_state_gather.cu", "fda_sched.cu", "fda_local_state_linear.cu", "fda_mean_state.cu", "fda_combine.cu", "fda_average.cu", "fda_noalloc.cu", "fda_probe.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC"]
 

@@ -343,11 +343,11 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     const float *xi_used = (flags & FDA_STATE_LINEAR) ? xi : nullptr;
     // With a list schedule in the context the cells can come from the list kernel.  In one pass over
-    // the K rows when there are few of them and the vector is long: 2.15 against 2.58 ms at 5 x 250,
+    // the K rows when there are few of them and the vector is long: 1.50 against 2.58 ms at 5 x 250,
     // K = 8, d = 198M, but no gain at d = 7M, where the averaged drifts and the 16-bit table of the
-    // two-pass route stay in L2.  From the averaged drifts that phase 1 leaves in memory when the
-    // sketch is too large for the lane-private bins of k_sketch_vector_rows: 1.02 against 1.42 ms at
-    // 7 x 500, K = 60, d = 20M (at 5 x 250 that kernel is the faster one: 0.22 against 0.25 ms at
+    // two-kernel route stay in L2.  From the averaged drifts that phase 1 below leaves in memory when
+    // the sketch is too large for the lane-private bins of k_sketch_vector_rows: 0.93 against 1.42 ms
+    // at 7 x 500, K = 60, d = 20M (at 5 x 250 that kernel is the faster one: 0.22 against 0.25 ms at
     // K = 30, d = 7M).
     const bool lists = sketch && ctx->sched != nullptr;
     const int64_t tiles = lists ? (d + ctx->sched_T - 1) / ctx->sched_T : 0;
