@@ -355,6 +355,7 @@ def run_ours(args, rank, world, local_rank):
         if it >= 3:
             mean_ms.append(e0.elapsed_time(e1))
     mean_ms = float(np.mean(mean_ms))
+    mean_kernel = ctx.fda_debug_last_kernel()
     mean_est = ctx.fda_combine_estimate(mean_state.view(1, -1), 1, F.FDA_VARIANT_SKETCH, eps, theta, est_buf).as_dict()
     # ---- a kernel that only reads, on the same tensor (yardstick for the streaming kernels) ----
     probe_out = torch.zeros(1, dtype=torch.float32, device=dev)
@@ -458,7 +459,8 @@ def run_ours(args, rank, world, local_rank):
             "mean_state": {"ms": mean_ms, "value": K * d / (mean_ms * 1e-3), "unit": UNIT,
                            "gbs": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9,
                            "frac_of_peak": 4.0 * (K * d + d + slen) / (mean_ms * 1e-3) / 1e9 / peak,
-                           "H": mean_est["H"], "note": "fda_mean_state: S-bar in one pass, no per-worker sketches"},
+                           "H": mean_est["H"], "kernel": mean_kernel,
+                           "note": "fda_mean_state: S-bar without the per-worker sketches"},
             "estimate": {"H": est.H, "trigger": int(est.trigger)},
             "roofline": roofline_of(run, peak, peak_kind),
             # what binds the sketch pass next to HBM: the shared-memory traffic of the l updates per
@@ -489,6 +491,17 @@ def run_ours(args, rank, world, local_rank):
         r4 = setup_and_time(4, max(3, min(args.steps, 20)), 3)
         r4.wl_id = 4
         p4 = r4.parts.mean(axis=0)
+        mean4 = torch.empty((r4.ctx.state_len,), dtype=torch.float32, device=dev)
+        mean4_ms = []
+        for it in range(3 + 10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            r4.ctx.fda_mean_state(r4.w_src[:, :r4.d], r4.w0_src, None, SKETCH_STATE, mean4)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                mean4_ms.append(e0.elapsed_time(e1))
+        mean4_ms = float(np.mean(mean4_ms))
         out["also"] = {
             "config": {"workload": "4:%s d=%d K=%d sketch=%dx%d eps=%.4f theta=%g" %
                                    (r4.wl.name, r4.d, r4.K, r4.wl.l, r4.wl.m, r4.wl.epsilon, r4.theta)},
@@ -501,6 +514,8 @@ def run_ours(args, rank, world, local_rank):
                              "frac_of_peak": 4.0 * (2 * r4.K * r4.d + r4.d) / (float(p4[2]) * 1e-3) / 1e9 / peak},
             "secondary_roofline": secondary_roofline(r4.ls_kernel, r4.K * r4.d * r4.wl.l / (float(p4[0]) * 1e-3), n_sm,
                                                      r4.clocks.get("sm_mhz") or 1965.0),
+            "mean_state": {"ms": mean4_ms, "value": r4.K * r4.d / (mean4_ms * 1e-3), "unit": UNIT,
+                           "kernel": r4.ctx.fda_debug_last_kernel()},
             "estimate": {"H": r4.est.H, "trigger": int(r4.est.trigger)},
             "context": {"device_bytes": r4.info["device_bytes"], "schedule_bytes": r4.info["schedule_bytes"],
                         "tile_indices": r4.info["tile_indices"], "fda_create_ms": r4.create_ms},

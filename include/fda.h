@@ -279,8 +279,8 @@ fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_hos
  * paper has no counterpart): "k_local_state_gather" (sketch pass over per-cell index lists: every sketch request
  * on a context that holds a list schedule), "k_local_state_linear" (no sketch requested),
  * "k_local_state_fast" / "k_local_state" (sketch requests without a schedule: aligned rows with 5
- * or 7 sketch rows / everything else); for fda_mean_state "k_local_state_gather(mean)" (one pass on
- * the list kernel), "k_mean_model + k_local_state_gather(mean)" (averaged drifts, then the list
+ * or 7 sketch rows / everything else); for fda_mean_state "k_mean_state_gather" (one pass on
+ * the list kernel), "k_mean_model + k_mean_state_gather" (averaged drifts, then the list
  * kernel on them), "k_mean_model + k_sketch_vector" (no schedule) or "k_mean_model" (no sketch
  * requested); "" before the first call.  The string is static;
  * ctx == NULL gives "".  Tests and the benchmark use it to say which kernel a number belongs to.

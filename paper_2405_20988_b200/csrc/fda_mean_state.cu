@@ -354,7 +354,7 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
     if (lists && K <= 2 * ctx->l && tiles >= 8 * (int64_t)ctx->n_sm) {
         const cudaError_t e = fda_launch_mean_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, mean_state, s);
         if (e != cudaErrorNotSupported) {
-            if (e == cudaSuccess) ctx->last_ls_kernel = "k_local_state_gather(mean)";
+            if (e == cudaSuccess) ctx->last_ls_kernel = "k_mean_state_gather";
             return e;
         }
     }
@@ -384,7 +384,7 @@ cudaError_t fda_launch_mean_state(fda_ctx *ctx, const float *w, int64_t row_stri
     if (lists && ctx->columns != 32) {
         e = fda_launch_mean_sketch_gather(ctx, ctx->mean_model, K, d, linear, flags, (int)nblk, mean_state, s);
         if (e != cudaErrorNotSupported) {
-            if (e == cudaSuccess) ctx->last_ls_kernel = "k_mean_model + k_local_state_gather(mean)";
+            if (e == cudaSuccess) ctx->last_ls_kernel = "k_mean_model + k_mean_state_gather";
             return e;
         }
     }

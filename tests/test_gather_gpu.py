@@ -221,8 +221,8 @@ def test_averaged_state_routes(env):
     rng = np.random.default_rng(27)
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     for K, d, l, m, want, lazy in [
-        (4, 6144 * 8 * n_sm + 13, 5, 250, "k_local_state_gather(mean)", False),
-        (20, 300_007, 7, 500, "k_mean_model + k_local_state_gather(mean)", True),
+        (4, 6144 * 8 * n_sm + 13, 5, 250, "k_mean_state_gather", False),
+        (20, 300_007, 7, 500, "k_mean_model + k_mean_state_gather", True),
     ]:
         coeffs = rand_coeffs(rng, l)
         w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
