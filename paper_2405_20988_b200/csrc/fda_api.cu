@@ -56,6 +56,9 @@ void free_device(fda_ctx *ctx)
     cudaFree(ctx->stage_xi);
     cudaFree(ctx->stage_states);
     cudaFree(ctx->stage_est);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
 }
 
 bool finite_f(float v) { return std::isfinite(v); }
@@ -123,6 +126,11 @@ fda_status fda_create_limited(fda_ctx **out, int device, int l, int m, const uin
             ctx->sched_build_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
         }
         if (e == cudaSuccess) e = cudaMalloc(&ctx->part_sk, sizeof(float) * ctx->part_sk_floats);
+        if (e == cudaSuccess && ctx->sched) {
+            e = cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+        }
     }
     ctx->part_np_doubles = (size_t)ctx->max_blocks * (size_t)(K_max > 32 ? K_max : 32) * 2;
     if (e == cudaSuccess) e = cudaMalloc(&ctx->part_np, sizeof(double) * ctx->part_np_doubles);

@@ -68,6 +68,9 @@ struct fda_ctx {
     int64_t sched_tiles = 0;
     double sched_build_ms = 0.0;      // host time spent building it
     float *mean_model = nullptr;      // d_max floats (average drift), allocated by the first fda_mean_state
+    // a second stream for the launches that fill the SMs the main launch of the list kernel leaves idle
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     double *combine_scratch = nullptr;        // 2 + FDA_MAX_ROWS doubles: S-bar[0..1] and the row norms
     unsigned int *combine_ticket = nullptr;   // blocks of the combine kernel that have finished (0 between launches)
     // staging for fda_round_host (lazy)

@@ -292,10 +292,19 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
     }
 }
 
+// The partial sums of a call come from up to three launches of the kernel (the main one and the
+// two that fill the SMs it leaves idle, see fda_launch_local_state_gather): launch q served the
+// groups g_first .. g_first + groups - 1 with cpg blocks each, block c * groups + (g - g_first)
+// writing slot slot_base + that number.
+struct ListParts {
+    int n;
+    int slot_base[3], g_first[3], groups[3], cpg[3];
+};
+
 // states[k][.] = sum of the partials of worker k's blocks in fp64, in a fixed order: four
 // adjacent lanes share one output, lane s adds the blocks s, s + 4, ... of the worker's group in
-// order (eight loads in flight), and the four sums are added as (s0 + s1) + (s2 + s3).
-__global__ void k_finalize_gather(const ListParams p, int blocks, uint32_t flags, float *__restrict__ states)
+// each launch in order (eight loads in flight), and the four sums are added as (s0 + s1) + (s2 + s3).
+__global__ void k_finalize_gather(const ListParams p, const ListParts parts, uint32_t flags, float *__restrict__ states)
 {
     const int lm = p.l * p.m, slen = 2 + lm;
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
@@ -310,26 +319,31 @@ __global__ void k_finalize_gather(const ListParams p, int blocks, uint32_t flags
         const int e = (int)((o / GW) % slen);
         const int g = (int)(o / ((int64_t)GW * slen));
         const int k = g * GW + kl;
-        const int nb = (blocks - g + p.groups - 1) / p.groups;        // blocks of this group: g, g + groups, ...
         double acc = 0.0;
-        if (!valid) {
-        } else if (e < 2) {
-            const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0
-                                     : ((flags & FDA_STATE_LINEAR) != 0 && p.have_xi);
-            if (on)
-                for (int j = sub; j < nb; j += 4) acc += p.part_np[((size_t)(g + j * p.groups) * GW + kl) * 2 + e];
-        } else if (sketch) {
-            const size_t step = (size_t)lm * GW * p.groups;             // from one block of the group to the next
-            const float *src = p.part_sk + (size_t)g * lm * GW + (size_t)(e - 2) * GW + kl + (size_t)sub * step;
-            int j = sub;
-            for (; j + 28 < nb; j += 32, src += 32 * step) {
-                float v[8];
+        for (int q = 0; q < parts.n; ++q) {
+            const int gl = g - parts.g_first[q];
+            if (!valid || gl < 0 || gl >= parts.groups[q]) continue;
+            const int nb = parts.cpg[q];                                // blocks of this group: gl, gl + groups, ...
+            const size_t first = (size_t)(parts.slot_base[q] + gl);
+            if (e < 2) {
+                const bool on = (e == 0) ? (flags & FDA_STATE_NORM) != 0
+                                         : ((flags & FDA_STATE_LINEAR) != 0 && p.have_xi);
+                if (on)
+                    for (int j = sub; j < nb; j += 4)
+                        acc += p.part_np[((first + (size_t)j * parts.groups[q]) * GW + kl) * 2 + e];
+            } else if (sketch) {
+                const size_t step = (size_t)lm * GW * parts.groups[q];  // from one block of the group to the next
+                const float *src = p.part_sk + first * lm * GW + (size_t)(e - 2) * GW + kl + (size_t)sub * step;
+                int j = sub;
+                for (; j + 28 < nb; j += 32, src += 32 * step) {
+                    float v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(4 * u) * step];
+                    for (int u = 0; u < 8; ++u) v[u] = src[(size_t)(4 * u) * step];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) acc += (double)v[u];
+                    for (int u = 0; u < 8; ++u) acc += (double)v[u];
+                }
+                for (; j < nb; j += 4, src += 4 * step) acc += (double)src[0];
             }
-            for (; j < nb; j += 4, src += 4 * step) acc += (double)src[0];
         }
         const double pair = acc + __shfl_xor_sync(0xffffffffu, acc, 1);      // lanes 0,1: s0 + s1; lanes 2,3: s2 + s3
         const double other = __shfl_xor_sync(0xffffffffu, pair, 2);
@@ -387,13 +401,66 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     // 8 producer + 20 walker warps, or 4 + 24 when a loaded index pays for more walking.  Measured:
     // 7 x 500, K = 60, d = 20M: 3.34 ms with 4 + 24 against 3.71 ms with 8 + 20; 5 x 250, K = 8,
     // d = 198M: 3.49 against 2.49 ms; 5 x 250, K = 30, d = 7M: 0.535 against 0.387 ms.
+    auto launch = [&](ListParams &q, int grid, cudaStream_t st) {
+        return ctx->l >= 7 ? launch_lists<4, 24>(q, grid, smem, ctx->smem_optin, st)
+                           : launch_lists<8, 20>(q, grid, smem, ctx->smem_optin, st);
+    };
+    ListParts parts{};
+    parts.n = 1;
+    parts.slot_base[0] = 0; parts.g_first[0] = 0; parts.groups[0] = p.groups; parts.cpg[0] = p.cpg;
+
+    // When the groups do not divide the SMs (K = 60: 15 groups x 9 blocks on 148 SMs) the SMs left
+    // over get the last tiles of every group, from the same kernel launched on a second stream with
+    // shifted pointers: first one block for each of the first `extra` groups, then the other groups
+    // on as many blocks each as fit.  The main launch stops at tile t1; all launches write their own
+    // slots of the partial sums.  Taken when the second of those launches still has a block per group
+    // and the job is long enough for the gain (tiles / cpg against t1 / cpg tile walks) to show.
+    const int extra = ctx->n_sm - blocks;
+    const int rest = p.groups - extra;                         // groups of the second tail launch (extra < groups)
+    int64_t t1 = p.tiles;
+    int cpg_b = 0;
+    if (extra > 0 && rest > 0 && extra / rest >= 1 && ctx->side_stream && p.tiles >= 64 * (int64_t)p.cpg) {
+        cpg_b = extra / rest;
+        // tail walks per block: n_tail + n_tail / cpg_b; main walks per block: (tiles - n_tail) / cpg
+        const double per_tail = 1.0 + 1.0 / (double)cpg_b;
+        int64_t n_tail = (int64_t)((double)p.tiles / (1.0 + (double)p.cpg * per_tail));
+        n_tail = n_tail / cpg_b * cpg_b;
+        const int64_t main_walks = (p.tiles - n_tail + p.cpg - 1) / p.cpg;
+        const size_t slots = (size_t)blocks + extra + (size_t)rest * cpg_b;
+        if (n_tail >= 4 * cpg_b && main_walks + 2 < (p.tiles + p.cpg - 1) / p.cpg &&
+            slots * ctx->lm * GW <= ctx->part_sk_floats && slots * GW * 2 <= ctx->part_np_doubles)
+            t1 = p.tiles - n_tail;
+    }
     cudaError_t e;
-    if (ctx->l >= 7) e = launch_lists<4, 24>(p, blocks, smem, ctx->smem_optin, s);
-    else e = launch_lists<8, 20>(p, blocks, smem, ctx->smem_optin, s);
+    if (t1 < p.tiles) {
+        const int64_t shift = t1 * p.T;                        // elements in front of the tail (a multiple of 1024)
+        ListParams ta = p;
+        ta.w = p.w + shift; ta.w_t0 = p.w_t0 + shift; ta.xi = p.xi ? p.xi + shift : nullptr;
+        ta.d = p.d - shift; ta.tiles = p.tiles - t1; ta.sched_off = p.sched_off + t1;
+        ListParams tb = ta;
+        ta.K = extra * GW; ta.groups = extra; ta.cpg = 1;
+        ta.part_sk = p.part_sk + (size_t)blocks * ctx->lm * GW; ta.part_np = p.part_np + (size_t)blocks * GW * 2;
+        tb.w = ta.w + (size_t)extra * GW * (size_t)row_stride; tb.K = K - extra * GW; tb.groups = rest; tb.cpg = cpg_b;
+        tb.part_sk = ta.part_sk + (size_t)extra * ctx->lm * GW; tb.part_np = ta.part_np + (size_t)extra * GW * 2;
+        parts.n = 3;
+        parts.slot_base[1] = blocks; parts.g_first[1] = 0; parts.groups[1] = extra; parts.cpg[1] = 1;
+        parts.slot_base[2] = blocks + extra; parts.g_first[2] = extra; parts.groups[2] = rest; parts.cpg[2] = cpg_b;
+        ListParams main = p;
+        main.tiles = t1; main.d = shift;
+        e = cudaEventRecord(ctx->ev_fork, s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0);
+        if (e == cudaSuccess) e = launch(ta, extra, ctx->side_stream);
+        if (e == cudaSuccess) e = launch(tb, rest * cpg_b, ctx->side_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_join, ctx->side_stream);
+        if (e == cudaSuccess) e = launch(main, blocks, s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ctx->ev_join, 0);
+    } else {
+        e = launch(p, blocks, s);
+    }
     if (e != cudaSuccess) return e;
     const int64_t total = (int64_t)p.groups * (2 + ctx->lm) * GW * 4;
     int fb = (int)((total + 255) / 256);
     if (fb > ctx->n_sm * 8) fb = ctx->n_sm * 8;
-    k_finalize_gather<<<fb, 256, 0, s>>>(p, blocks, flags, states);
+    k_finalize_gather<<<fb, 256, 0, s>>>(p, parts, flags, states);
     return cudaGetLastError();
 }

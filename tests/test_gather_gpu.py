@@ -174,6 +174,15 @@ def test_sixty_workers_seven_by_five_hundred_run_on_the_list_kernel(env):
     run(env, 58, 700_001, 7, 500, seed=24, flags=1 | 4, workers=[0, 55, 57])      # last group: two workers
 
 
+def test_groups_that_do_not_divide_the_sms_use_the_tail_launches(env):
+    """Fifteen worker groups on nine blocks each leave SMs idle; on long vectors those get the last
+    tiles of every group through two more launches of the kernel (one block per group for the first
+    groups, the other groups after them).  Workers of both tail launches, of the last (partial)
+    group, and a ragged last tile."""
+    run(env, 60, 3_000_017, 7, 500, seed=28, workers=[0, 3, 51, 52, 55, 59])
+    run(env, 58, 3_100_003, 7, 500, seed=29, flags=1 | 4, workers=[1, 50, 53, 56, 57])
+
+
 def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
     torch, oracle, F = env
     rng = np.random.default_rng(25)
