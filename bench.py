@@ -245,6 +245,7 @@ def run_ours(args, rank, world, local_rank):
         r.est_buf = ctx.new_estimate_buffer(dev)
         r.theta, r.eps = float(wl.thetas[-1]), float(np.float32(wl.epsilon))
         r.ls_kernel = ""       # the kernel the library picked for the sketch pass (asked after each launch)
+        r.ls_launches = 2
         w, w0, states, est_buf = r.w, r.w0, r.states, r.est_buf
 
         def step_events():
@@ -252,6 +253,7 @@ def run_ours(args, rank, world, local_rank):
             ev[0].record(stream)
             ctx.fda_local_state(w[:, :d], w0, None, SKETCH_STATE, states)
             r.ls_kernel = ctx.fda_debug_last_kernel()
+            r.ls_launches = ctx.fda_debug_last_launches()
             ev[1].record(stream)
             ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, r.eps, r.theta, est_buf, want_host=False)
             ev[2].record(stream)
@@ -472,7 +474,7 @@ def run_ours(args, rank, world, local_rank):
             "e2e": None if not e2e_times else
                    {"value": job_value(world, K * d, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "api": "fda_round_host"},
-            "gpu_launches": 4 * args.steps,
+            "gpu_launches": (run.ls_launches + 2) * args.steps,     # the state pass, its finalize, combine, average
             "clocks": clocks,
             "context": {"device_bytes": run.info["device_bytes"], "schedule_bytes": run.info["schedule_bytes"],
                         "tile_indices": run.info["tile_indices"], "table_bytes": run.info["table_bytes"],
@@ -521,7 +523,7 @@ def run_ours(args, rank, world, local_rank):
                         "tile_indices": r4.info["tile_indices"], "fda_create_ms": r4.create_ms},
             "clocks": r4.clocks,
         }
-        out["gpu_launches"] += 4 * int(r4.parts.shape[0])
+        out["gpu_launches"] += (r4.ls_launches + 2) * int(r4.parts.shape[0])
         r4.ctx.close()
     if dist:
         dist.barrier()

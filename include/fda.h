@@ -288,6 +288,15 @@ fda_status fda_debug_schedule(const fda_ctx *ctx, int64_t tile, void *record_hos
 const char *fda_debug_last_kernel(const fda_ctx *ctx);
 
 /*
+ * Number of kernels the context's last fda_local_state call launched (the paper has no
+ * counterpart): 2 (the pass and the kernel that adds up its per-block partial sums), or 4 when the
+ * sketch pass over index lists also ran its two tail launches on the context's second stream (worker
+ * groups that do not divide the SMs, long vectors).  0 before the first call or for ctx == NULL.
+ * The benchmark uses it to count the launches of a step.
+ */
+int fda_debug_last_launches(const fda_ctx *ctx);
+
+/*
  * Local state without a context and without any allocation.  (The paper has no counterpart
  * to this call; it exists for the way some programs have to use the library.)
  *

@@ -21,7 +21,7 @@ _STATUS = {0: "FDA_OK", 1: "FDA_ERR_INVALID_ARG", 2: "FDA_ERR_UNSUPPORTED", 3: "
            4: "FDA_ERR_NOMEM"}
 
 EXPORTS = ("fda_create", "fda_create_limited", "fda_context_info", "fda_destroy", "fda_state_len", "fda_last_error", "fda_local_state", "fda_mean_state",
-           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel", "fda_debug_schedule",
+           "fda_combine_estimate", "fda_average_models", "fda_average_models_xi", "fda_round_host", "fda_debug_hash", "fda_debug_read_probe", "fda_debug_last_kernel", "fda_debug_last_launches", "fda_debug_schedule",
            "fda_local_state_linear_noalloc")
 FDA_NOALLOC_MAX_WORKERS = 64
 
@@ -87,6 +87,8 @@ def load_library():
     lib.fda_debug_schedule.restype = c_int
     lib.fda_debug_last_kernel.argtypes = [vp]
     lib.fda_debug_last_kernel.restype = ctypes.c_char_p
+    lib.fda_debug_last_launches.argtypes = [vp]
+    lib.fda_debug_last_launches.restype = ctypes.c_int
     lib.fda_local_state_linear_noalloc.argtypes = [c_int, vp, i64, c_int, i64, vp, vp, u32, vp, vp]
     lib.fda_local_state_linear_noalloc.restype = c_int
     for name in ("fda_create", "fda_destroy", "fda_local_state", "fda_combine_estimate",
@@ -306,6 +308,10 @@ class FdaContext:
     def fda_debug_last_kernel(self) -> str:
         """Name of the kernel that served the last fda_local_state call on this context."""
         return self._lib.fda_debug_last_kernel(self._h).decode()
+
+    def fda_debug_last_launches(self) -> int:
+        """Kernels that the last fda_local_state call on this context launched."""
+        return int(self._lib.fda_debug_last_launches(self._h))
 
     @staticmethod
     def new_estimate_buffer(device="cuda"):

@@ -165,6 +165,8 @@ const char *fda_last_error(const fda_ctx *ctx) { return ctx ? ctx->err.c_str() :
 
 const char *fda_debug_last_kernel(const fda_ctx *ctx) { return ctx ? ctx->last_ls_kernel : ""; }
 
+int fda_debug_last_launches(const fda_ctx *ctx) { return ctx ? ctx->last_ls_launches : 0; }
+
 fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                            const float *w_t0, const float *xi, uint32_t flags, float *states,
                            void *stream)

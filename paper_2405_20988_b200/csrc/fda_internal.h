@@ -79,6 +79,7 @@ struct fda_ctx {
     int64_t stage_stride = 0;
     uint64_t coeffs_host[6 * FDA_MAX_ROWS] = {0};
     const char *last_ls_kernel = "";   // which kernel served the last fda_local_state / fda_mean_state
+    int last_ls_launches = 0;          // kernels the last fda_local_state launched
     std::string err;
 };
 

@@ -468,15 +468,16 @@ cudaError_t fda_launch_local_state(fda_ctx *ctx, const float *w, int64_t row_str
     {   // sketch requests: the list kernel when the context holds its schedule; requests without a
         // sketch: the streaming kernel; everything else: the plain-load kernels below
         cudaError_t e = fda_launch_local_state_gather(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_gather"; return e; }
+        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_gather"; return e; }   // (counts its launches itself)
         e = fda_launch_local_state_linear(ctx, w, row_stride, K, d, w_t0, xi, flags, states, s);
-        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_linear"; return e; }
+        if (e != cudaErrorNotSupported) { ctx->last_ls_kernel = "k_local_state_linear"; ctx->last_ls_launches = 2; return e; }
     }
     if (flags & FDA_STATE_SKETCH) {
         const cudaError_t e = fda_ensure_table(ctx, s);
         if (e != cudaSuccess) return e;
     }
     ctx->last_ls_kernel = "k_local_state";
+    ctx->last_ls_launches = 2;
     const bool sketch = (flags & FDA_STATE_SKETCH) != 0;
     LsParams p{};
     p.w = w; p.row_stride = row_stride; p.K = K; p.d = d; p.w_t0 = w_t0;

@@ -462,5 +462,6 @@ cudaError_t fda_launch_local_state_gather(fda_ctx *ctx, const float *w, int64_t 
     int fb = (int)((total + 255) / 256);
     if (fb > ctx->n_sm * 8) fb = ctx->n_sm * 8;
     k_finalize_gather<<<fb, 256, 0, s>>>(p, parts, flags, states);
+    ctx->last_ls_launches = parts.n + 1;
     return cudaGetLastError();
 }

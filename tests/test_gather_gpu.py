@@ -38,7 +38,7 @@ def rand_coeffs(rng, l):
     return c
 
 
-def run(env, K, d, l, m, seed, flags=ALL, misalign=0, coeffs=None, sigma=1e-3, workers=None, expect=GATHER):
+def run(env, K, d, l, m, seed, flags=ALL, misalign=0, coeffs=None, sigma=1e-3, workers=None, expect=GATHER, launches=2):
     torch, oracle, F = env
     rng = np.random.default_rng(seed)
     stride = S.row_stride(d)
@@ -59,6 +59,7 @@ def run(env, K, d, l, m, seed, flags=ALL, misalign=0, coeffs=None, sigma=1e-3, w
         ctx.fda_local_state(w[:, :d], w0, xg, flags, st)
         torch.cuda.synchronize()
         name = ctx.fda_debug_last_kernel()
+        assert ctx.fda_debug_last_launches() == launches
         got = st.cpu().numpy()
     if expect is not None:
         assert name == expect, name
@@ -179,8 +180,8 @@ def test_groups_that_do_not_divide_the_sms_use_the_tail_launches(env):
     tiles of every group through two more launches of the kernel (one block per group for the first
     groups, the other groups after them).  Workers of both tail launches, of the last (partial)
     group, and a ragged last tile."""
-    run(env, 60, 3_000_017, 7, 500, seed=28, workers=[0, 3, 51, 52, 55, 59])
-    run(env, 58, 3_100_003, 7, 500, seed=29, flags=1 | 4, workers=[1, 50, 53, 56, 57])
+    run(env, 60, 3_000_017, 7, 500, seed=28, workers=[0, 3, 51, 52, 55, 59], launches=4)
+    run(env, 58, 3_100_003, 7, 500, seed=29, flags=1 | 4, workers=[1, 50, 53, 56, 57], launches=4)
 
 
 def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
