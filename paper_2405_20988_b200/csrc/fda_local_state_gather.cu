@@ -57,6 +57,11 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
     constexpr int kThreads = (PW + WW) * 32;
     constexpr int kBatch = PW * 32 * 4;                       // a batch is four consecutive indices per producer thread
     constexpr int kDepth = 1;                                 // batches a producer thread keeps in flight
+    // entry chunks (four steps each) a walker loads before it walks them: eight, or five with the
+    // 4 + 24 split, whose items average eleven steps (7 x 500, K = 60, d = 20M: 2.94 ms with 5, 2.98
+    // with 4, 2.96 with 6, 3.01 with 7, 3.06 with 8; 5 x 250, K = 8, d = 198M with 8 + 20 warps: 2.48 ms
+    // with 8, 2.47 with 7, 2.51 with 6, 2.52 with 10)
+    constexpr int kAhead = (WW == 24) ? 5 : kChunksAhead;
     static_assert(PW <= kMaxProducerWarps, "the fp64 sums have room for kMaxProducerWarps warps");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -238,15 +243,15 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
                 const uint2 *ent = reinterpret_cast<const uint2 *>(ent0 + (size_t)chunk0 * 256) + lane;
                 const int nch = (steps + 3) >> 2;
                 unsigned long long a01 = 0ull, a23 = 0ull;
-                // all entry loads of (up to) eight chunks first, then the walk: the entries come
-                // from global memory (L2), one round trip per eight chunks instead of one per chunk
-                for (int c0 = 0; c0 < nch; c0 += kChunksAhead) {
-                    uint2 ch[kChunksAhead];
+                // all entry loads of (up to) kAhead chunks first, then the walk: the entries come
+                // from global memory (L2), one round trip per kAhead chunks instead of one per chunk
+                for (int c0 = 0; c0 < nch; c0 += kAhead) {
+                    uint2 ch[kAhead];
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q)
+                    for (int q = 0; q < kAhead; ++q)
                         if (c0 + q < nch) ch[q] = __ldg(ent + (size_t)(c0 + q) * kListSlots);
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q) {
+                    for (int q = 0; q < kAhead; ++q) {
                         const int left = steps - 4 * (c0 + q);
                         if (left >= 4) {
                             gather_lo(ch[q].x, base, a01, a23);

@@ -111,7 +111,9 @@ inline size_t mean_smem_fixed(int l, int m, int T, int tab_bytes)
 //   then        ut[2][T + 8]   (summed drifts; eight zero rows behind each)
 //   then        the landing zone: depth slots of R rows of kRowPitch bytes
 // (each region on a 128-byte boundary)
-template <bool LINEAR>
+// AHEAD: entry chunks (four steps each) a walker loads before it walks them (five for sketches of
+// seven or more rows, whose items are short; else eight - as in k_local_state_gather).
+template <bool LINEAR, int AHEAD>
 __global__ void __launch_bounds__(kThreads, 1) k_mean_state_gather(const MeanParams mp)
 {
     const ListParams &p = mp.q;
@@ -275,14 +277,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_mean_state_gather(const MeanPar
                 const uint2 *ent = reinterpret_cast<const uint2 *>(ent0 + (size_t)chunk0 * 256) + lane;
                 const int nch = (steps + 3) >> 2;
                 float a = 0.f;
-                // all entry loads of (up to) eight chunks first, then the walk
-                for (int c0 = 0; c0 < nch; c0 += kChunksAhead) {
-                    uint2 ch[kChunksAhead];
+                // all entry loads of (up to) AHEAD chunks first, then the walk
+                for (int c0 = 0; c0 < nch; c0 += AHEAD) {
+                    uint2 ch[AHEAD];
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q)
+                    for (int q = 0; q < AHEAD; ++q)
                         if (c0 + q < nch) ch[q] = __ldg(ent + (size_t)(c0 + q) * kListSlots);
 #pragma unroll
-                    for (int q = 0; q < kChunksAhead; ++q) {
+                    for (int q = 0; q < AHEAD; ++q) {
                         const int left = steps - 4 * (c0 + q);
                         if (left >= 4) {
                             gather1(ch[q].x & 0xffffu, base, a);
@@ -398,7 +400,8 @@ cudaError_t launch_mean(fda_ctx *ctx, const float *w, int64_t row_stride, int ro
     mp.depth = (int)(depth < (size_t)kMaxDepth ? depth : (size_t)kMaxDepth);
     const size_t smem = fixed + (size_t)mp.depth * per_quad;
 
-    auto kern = xi_used ? k_mean_state_gather<true> : k_mean_state_gather<false>;
+    auto kern = ctx->l >= 7 ? (xi_used ? k_mean_state_gather<true, 5> : k_mean_state_gather<false, 5>)
+                            : (xi_used ? k_mean_state_gather<true, kChunksAhead> : k_mean_state_gather<false, kChunksAhead>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin);
     if (e != cudaSuccess) return e;
     kern<<<blocks, kThreads, smem, s>>>(mp);
