@@ -8,7 +8,7 @@
 namespace fda_list {
 
 constexpr int GW = kListWorkers;
-constexpr int kChunksAhead = 8;                // entry chunks (four steps each) a walker loads before it walks them
+constexpr int kChunksAhead = 8;                // entry chunks (four steps each) the walkers of the averaged state load ahead (sketches below 7 rows)
 constexpr int kMaxProducerWarps = 16;          // the fp64 sums in shared memory have room for that many
 
 struct ListParams {

@@ -57,11 +57,11 @@ __global__ void __launch_bounds__((PW + WW) * 32, 1) k_local_state_gather(const 
     constexpr int kThreads = (PW + WW) * 32;
     constexpr int kBatch = PW * 32 * 4;                       // a batch is four consecutive indices per producer thread
     constexpr int kDepth = 1;                                 // batches a producer thread keeps in flight
-    // entry chunks (four steps each) a walker loads before it walks them: eight, or five with the
-    // 4 + 24 split, whose items average eleven steps (7 x 500, K = 60, d = 20M: 2.94 ms with 5, 2.98
-    // with 4, 2.96 with 6, 3.01 with 7, 3.06 with 8; 5 x 250, K = 8, d = 198M with 8 + 20 warps: 2.48 ms
-    // with 8, 2.47 with 7, 2.51 with 6, 2.52 with 10)
-    constexpr int kAhead = (WW == 24) ? 5 : kChunksAhead;
+    // entry chunks (four steps each) a walker loads before it walks them: seven (items of 5 x 250
+    // average 28 steps), or five with the 4 + 24 split, whose items average eleven steps.  Measured:
+    // 7 x 500, K = 60, d = 20M: 2.94 ms with 5, 2.98 with 4, 2.96 with 6, 3.01 with 7, 3.06 with 8;
+    // 5 x 250, K = 8, d = 198M with 8 + 20 warps: 2.474 ms with 7, 2.481 with 8, 2.51 with 6, 2.52 with 10
+    constexpr int kAhead = (WW == 24) ? 5 : 7;
     static_assert(PW <= kMaxProducerWarps, "the fp64 sums have room for kMaxProducerWarps warps");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
