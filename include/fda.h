@@ -144,6 +144,10 @@ const char *fda_last_error(const fda_ctx *ctx);
  * or > d_max, row_stride < d, unknown flag, SKETCH without a sketch), UNSUPPORTED (more worker
  * groups than the context's partial-sum scratch holds: K above 4 x the SM count with a list
  * schedule, above 32 x the SM count without; nothing is launched), CUDA.
+ * Stream order: the call's work starts after what `stream` held before it and is complete before
+ * anything enqueued on `stream` after it.  Part of it may run on a second stream that the context
+ * owns (forked from and joined to `stream` with events; also legal while `stream` is being
+ * captured into a graph), which is why a context serves one stream at a time.
  */
 fda_status fda_local_state(fda_ctx *ctx, const float *w, int64_t row_stride, int K, int64_t d,
                            const float *w_t0, const float *xi, uint32_t flags, float *states,

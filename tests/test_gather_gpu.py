@@ -184,6 +184,45 @@ def test_groups_that_do_not_divide_the_sms_use_the_tail_launches(env):
     run(env, 58, 3_100_003, 7, 500, seed=29, flags=1 | 4, workers=[1, 50, 53, 56, 57], launches=4)
 
 
+def test_a_round_with_tail_launches_can_be_captured_in_a_graph(env):
+    """fda_local_state forks to the context's second stream and joins again with events: legal while
+    the caller's stream is being captured.  The replayed graph (local state, estimate, average) gives
+    the bits of the eager calls - every reduction of the path has a fixed order."""
+    torch, oracle, F = env
+    rng = np.random.default_rng(30)
+    K, d, l, m = 60, 3_000_017, 7, 500
+    w_src = (torch.randn((K, d), device="cuda") * 1e-3)
+    w0_src = torch.randn(d, device="cuda") * 0.05
+    w_src += w0_src
+    with F.FdaContext(l, m, rand_coeffs(rng, l), d_max=d, K_max=K) as ctx:
+        def round_(w, w0, states, est):
+            ctx.fda_local_state(w, w0, None, 1 | 4, states)
+            ctx.fda_combine_estimate(states, K, F.FDA_VARIANT_SKETCH, 0.0424, 1e-6, est, want_host=False)
+            ctx.fda_average_models(w, w0, est, F.FDA_AVG_BROADCAST)
+        w, w0 = w_src.clone(), w0_src.clone()
+        st_e = torch.zeros((K, ctx.state_len), device="cuda")
+        est_e = ctx.new_estimate_buffer()
+        round_(w, w0, st_e, est_e)
+        assert ctx.fda_debug_last_launches() == 4
+        torch.cuda.synchronize()
+        w_e, w0_e = w.clone(), w0.clone()
+        w.copy_(w_src); w0.copy_(w0_src)
+        st_g = torch.zeros_like(st_e)
+        est_g = ctx.new_estimate_buffer()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            round_(w, w0, st_g, est_g)
+        for _ in range(2):                      # the captured round, twice, from the same inputs
+            w.copy_(w_src); w0.copy_(w0_src); st_g.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(st_g, st_e)
+            assert bytes(est_g.cpu().numpy()) == bytes(est_e.cpu().numpy())
+            assert torch.equal(w, w_e) and torch.equal(w0, w0_e)
+            assert float(w_e[0, 0]) != float(w_src[0, 0])      # the round did synchronise
+
+
 def test_context_reports_its_footprint_and_the_schedule_can_be_capped(env):
     torch, oracle, F = env
     rng = np.random.default_rng(25)
