@@ -76,3 +76,36 @@ def test_rounds_follow_the_oracle(variant, theta, refresh, averaged):
         assert got["syncs"] == list(range(steps))        # Theta = 0 is the Synchronous scheme
     if theta == 1e9:
         assert got["syncs"] == []
+
+
+@pytest.mark.parametrize("variant,refresh,averaged", [(1, False, False), (1, False, True), (0, True, False)])
+def test_rounds_replayed_from_a_graph_give_the_eager_bits(variant, refresh, averaged):
+    """graph=True records the library calls of a step once and replays them: the same estimates,
+    synchronisation steps, account and final models, bit for bit, as the eager loop."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("CUDA device required for -m gpu tests")
+    import paper_2405_20988_b200 as F
+
+    rng = np.random.default_rng(78)
+    K, d, l, m, steps, eps, theta = 6, 20_011, 5, 250, 14, 0.06, 2e-3
+    coeffs = S.hash_coefficients(6, l)
+    w_t0 = rng.normal(0, 0.05, size=d).astype(np.float32)
+    xi = rng.normal(size=d)
+    xi = (xi / np.linalg.norm(xi)).astype(np.float32)
+    common = rng.normal(0, 2e-4, size=(steps, 1, d)).astype(np.float32)
+    dev = torch.from_numpy((common + rng.normal(0, 2e-4, size=(steps, K, d))).astype(np.float32)).cuda()
+    results = []
+    for graph in (False, True):
+        with F.FdaContext(l, m, coeffs, d_max=d, K_max=K) as ctx:
+            w = torch.from_numpy(np.tile(w_t0, (K, 1))).cuda()
+            w0 = torch.from_numpy(w_t0.copy()).cuda()
+            xg = torch.from_numpy(xi.copy()).cuda()
+            got = F.run_rounds(ctx, w, w0, xg, steps, lambda t, ww: ww.add_(dev[t]), variant, eps, theta,
+                               refresh_xi=refresh, averaged_state=averaged, graph=graph)
+            torch.cuda.synchronize()
+            results.append((got, w.cpu().numpy(), w0.cpu().numpy(), xg.cpu().numpy()))
+    (a, wa, w0a, xa), (b, wb, w0b, xb) = results
+    assert a["H"] == b["H"] and a["syncs"] == b["syncs"] and 0 < len(a["syncs"]) < steps
+    assert a["state_bytes"] == b["state_bytes"] and a["model_bytes"] == b["model_bytes"]
+    assert np.array_equal(wa, wb) and np.array_equal(w0a, w0b) and np.array_equal(xa, xb)
