@@ -209,7 +209,7 @@ def test_heavy_tailed_values(env):
 @pytest.mark.parametrize("K,d,l,m,misalign", [
     (1, 1, 5, 250, 0), (2, 7, 3, 7, 0), (5, 4099, 5, 250, 0), (8, 100_003, 5, 250, 0), (30, 20_001, 5, 250, 0),
     (60, 30_011, 7, 500, 0), (9, 9_999, 16, 1000, 0), (13, 10_007, 5, 250, 3), (4, 3_000, 2, 20_000, 0),
-    (6, 40_000, 3, 100, 0), (18, 100_001, 7, 500, 1),
+    (6, 40_000, 3, 100, 0), (18, 100_001, 7, 500, 1), (20, 100, 7, 500, 0), (3, 5, 7, 500, 1), (2, 5121, 7, 500, 0),
     # long vectors with few workers: the one-pass route on the list kernel (it needs eight tiles per SM)
     (3, 7_400_003, 5, 250, 0), (5, 7_300_001, 5, 250, 1), (10, 7_280_000, 5, 250, 0),
 ])
